@@ -1,0 +1,218 @@
+/*
+ * saem.h -- C ABI of the B200 (sm_100a) MoE expert-step library.
+ *
+ * One MoE layer step of a stage-aware MoE decoding runtime:
+ *
+ *   saem_route      top-k gating                         (Background, "Mixture-of-Experts Inference")
+ *   saem_repack     expert-aligned token repacking       (Sec. IV-E)
+ *   saem_expert_ffn grouped SwiGLU expert FFN over the   (Sec. IV-E "single batched launch per expert",
+ *                   repacked segments, weights read from  Sec. IV-C fixed-size expert cache region)
+ *                   an HBM expert-slot cache
+ *   saem_combine    weighted merge back to token order   (Sec. IV-D, merge of expert outputs)
+ *   saem_cache_*    expert-slot table: asynchronous       (Sec. IV-C "Latency-Hiding Prefetch and Overlap",
+ *                   host->HBM loads with events, evict     residency map + fixed per-layer slot layout)
+ *
+ * General conventions
+ *   - Plain C.  Streams are passed as `void*` holding a cudaStream_t (NULL = the legacy default stream).
+ *   - "dev" pointers are CUDA device pointers, "host" pointers ordinary host memory, "pinned" host
+ *     memory registered with CUDA (cudaHostAlloc / cudaHostRegister).  All device buffers are owned
+ *     by the caller, must be 16-byte aligned (slot region and workspace: 1024-byte aligned) and
+ *     must stay valid until the work enqueued on them has finished.
+ *   - The library allocates no device memory.  It owns only host tables and CUDA events.
+ *   - bf16 tensors are raw 16-bit patterns; every matrix is row-major; pair id p = t*top_k + j.
+ *   - Every function returns a saem_status.  Errors a host can see (bad argument, shape, alignment,
+ *     residency) are returned before anything is enqueued.  Conditions only the device can see
+ *     (a routed expert that is not resident when no subset was given, an index out of range, a
+ *     bounded wait that ran out) set a sticky device status word, read by
+ *     saem_last_device_status(); kernels never trap and never wait without a bound.
+ *   - The four step calls never synchronise and never read device results on the host.
+ */
+#ifndef SAEM_H_
+#define SAEM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct saem_ctx saem_ctx;   /* opaque: host tables, events, workspace carving */
+
+typedef enum saem_status {
+    SAEM_OK = 0,
+    SAEM_ERR_INVALID_ARG = 1,
+    SAEM_ERR_SHAPE = 2,
+    SAEM_ERR_ALIGNMENT = 3,
+    SAEM_ERR_WORKSPACE = 4,
+    SAEM_ERR_NOT_RESIDENT = 5,
+    SAEM_ERR_SLOT_BUSY = 6,
+    SAEM_ERR_TIMEOUT = 7,
+    SAEM_ERR_CUDA = 8,
+    SAEM_ERR_UNSUPPORTED = 9
+} saem_status;
+
+enum { SAEM_MAX_EXPERTS = 128 };         /* routed experts per layer */
+enum { SAEM_TEMP = -2 };                 /* slot argument of saem_cache_load: take a temporary slot */
+enum { SAEM_OUT_F32 = 0, SAEM_OUT_BF16 = 1 };
+enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2 };
+
+/*
+ * Shape of one context.  d_model and d_ff must be multiples of 128; 1 <= top_k <= n_experts <=
+ * SAEM_MAX_EXPERTS; max_tokens * top_k <= 65535.  The slot region holds n_layers * slots_per_layer
+ * fixed slots (slot s of layer l is global slot l * slots_per_layer + s) followed by temp_slots
+ * temporary slots shared by all layers (Sec. VI ablation: on-demand loads through a reserved
+ * temporary slot).  renorm: 1 = softmax over the k selected logits (weights sum to 1), 0 = the
+ * selected experts' probabilities under the softmax over all experts.  out_dtype: SAEM_OUT_*.
+ * ffn_path: SAEM_FFN_AUTO picks the tensor-core streaming kernels; SAEM_FFN_SCALAR forces the
+ * plain scalar kernels (kept for triage).
+ */
+typedef struct saem_config {
+    int32_t d_model;
+    int32_t d_ff;
+    int32_t n_experts;
+    int32_t top_k;
+    int32_t max_tokens;
+    int32_t n_layers;
+    int32_t slots_per_layer;
+    int32_t temp_slots;
+    int32_t renorm;
+    int32_t out_dtype;
+    int32_t ffn_path;
+    int32_t reserved;
+} saem_config;
+
+/* Library version (major*10000 + minor*100 + patch) and a static string for a status code. */
+int saem_version(void);
+const char* saem_status_string(int status);
+
+/* Bytes of one packed expert (= one slot): 3 * d_model * d_ff * 2.  0 on an invalid config. */
+size_t saem_slot_bytes(const saem_config* cfg);
+/* Bytes the slot region must have: (n_layers * slots_per_layer + temp_slots) * saem_slot_bytes. */
+size_t saem_slot_region_bytes(const saem_config* cfg);
+/* Bytes of device workspace a context needs (hidden activations h[max_tokens*top_k, d_ff] in
+ * bf16, split-K partial tiles and counters, the device status word, and the buffers of
+ * saem_moe_step).  Allocated once by the caller and reused by every layer (Sec. IV-E). */
+size_t saem_workspace_bytes(const saem_config* cfg);
+
+/*
+ * Create a context over caller-owned device memory.  Both regions must be 1024-byte aligned and at
+ * least as large as the two size queries say.  The workspace is cleared by an asynchronous memset
+ * on the legacy default stream followed by a synchronisation; all slots start empty.  The current
+ * CUDA device at the time of the call is the context's device.
+ * Errors: INVALID_ARG (null), SHAPE (config limits), ALIGNMENT, WORKSPACE (too small), CUDA.
+ */
+int saem_create(const saem_config* cfg, void* dev_slot_region, size_t slot_region_bytes,
+                void* dev_workspace, size_t workspace_bytes, saem_ctx** out);
+void saem_destroy(saem_ctx* ctx);
+
+/*
+ * One-time, offline: rewrite one expert from the canonical layout (gate[d_ff, d_model],
+ * up[d_ff, d_model], down[d_model, d_ff], row-major bf16, host memory) into the slot layout
+ * (host memory, saem_slot_bytes): tiles of 128 weight rows x 64 reduction elements, each tile
+ * 16 KB with its 16-byte chunks XOR-swizzled by (row mod 8) so that a tile can be bulk-copied
+ * into shared memory and fed to the tensor cores as is; gate and up tiles of the same position
+ * are adjacent.  A slot's content is opaque to the caller.
+ */
+int saem_pack_expert_host(const saem_config* cfg, const void* gate, const void* up, const void* down,
+                          void* packed_out);
+
+/*
+ * Top-k gating.  logits[T, n_experts] fp32 (dev) -> topk_idx[T, top_k] int32, topk_w[T, top_k] fp32
+ * (dev).  Slot j of a token holds its j-th largest logit: k rounds of arg-max comparing (value
+ * descending, expert id ascending); NaN counts as -inf; +0 == -0.  Weights per config.renorm,
+ * computed in fp32 with the row maximum subtracted.  A row whose best logit is -inf gets 1/k
+ * everywhere; +inf logits share the weight equally.  Errors: SHAPE if T < 0 or T > max_tokens.
+ * T == 0 is a no-op.
+ */
+int saem_route(saem_ctx* ctx, const float* logits, int T, int32_t* topk_idx, float* topk_w, void* stream);
+
+/*
+ * Expert-aligned token repacking.  topk_idx[T, top_k] (dev) and x[T, d_model] bf16 (dev) ->
+ * counts[n_experts], offsets[n_experts + 1] (exclusive scan, offsets[E] = T*top_k), perm[T*top_k]
+ * (pair stored at packed row r), inv_perm[T*top_k] (packed row of pair p), x_packed[T*top_k,
+ * d_model] bf16 = x[perm[r] / top_k].  Segments are in ascending expert id and keep ascending pair
+ * id inside (a stable counting sort), so the permutation is unique.  An index outside
+ * [0, n_experts) sets the device status word and the pair is dropped from every output.
+ */
+int saem_repack(saem_ctx* ctx, const int32_t* topk_idx, const void* x, int T, int32_t* counts,
+                int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* x_packed, void* stream);
+
+/*
+ * Grouped SwiGLU expert FFN.  For every expert e with rows r in [offsets[e], offsets[e+1]) of
+ * x_packed (dev, bf16): y_packed[r] = Wd_e * ( silu(Wg_e * x_r) .* (Wu_e * x_r) ), fp32
+ * accumulation, hidden activations rounded to bf16 in the context's workspace, y_packed[max_rows,
+ * d_model] fp32 (dev).  Weights come from the slots that `layer`'s residency map (or a temporary
+ * slot) gives.  offsets (dev) is read on the device only; max_rows bounds offsets[n_experts] and
+ * must not exceed max_tokens * top_k.
+ *   expert_subset (host, may be NULL): run only these experts (rows of the others are left
+ *   untouched).  With a subset, an expert that has no slot returns NOT_RESIDENT before any
+ *   enqueue.  Without one, experts without a slot are skipped on the device; if such an expert has
+ *   rows, the device status word becomes NOT_RESIDENT and its rows are left untouched.
+ * If a needed slot's load is still in flight on another stream, `stream` is made to wait for its
+ * completion event first.
+ */
+int saem_expert_ffn(saem_ctx* ctx, int layer, const void* x_packed, const int32_t* offsets, int max_rows,
+                    const int32_t* expert_subset, int n_subset, float* y_packed, void* stream);
+
+/*
+ * Weighted merge: out[t] = sum_{j = 0..top_k-1, in that order} topk_w[t, j] *
+ * y_packed[inv_perm[t*top_k + j]] (+ shared_y[t] if not NULL, fp32 [T, d_model], added last).
+ * Gather-based, no atomics: two runs give identical bits.  out[T, d_model] fp32 or bf16 per
+ * config.out_dtype.
+ */
+int saem_combine(saem_ctx* ctx, const float* y_packed, const int32_t* inv_perm, const float* topk_w, int T,
+                 const float* shared_y, void* out, void* stream);
+
+/*
+ * The whole layer step on device buffers: route -> repack -> expert FFN -> [shared expert FFN via
+ * shared_ctx over x itself] -> combine, enqueued on `stream`, intermediates in ctx's workspace.
+ * shared_ctx (may be NULL) is a context with n_experts = top_k = 1 whose layer `layer` slot 0
+ * holds the always-on shared expert (two shared experts of width f are packed as one of width 2f).
+ * logits[T, E] fp32, x[T, d] bf16, out[T, d] (all dev).
+ */
+int saem_moe_step(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const float* logits, const void* x, int T,
+                  void* out, void* stream);
+
+/*
+ * The same step from HOST buffers (pinned memory recommended): copies logits and x to the device,
+ * runs saem_moe_step, copies out back and synchronises `stream`.  Expert weights stay in the HBM
+ * slots.  logits_host[T, E] fp32, x_host[T, d] bf16, out_host[T, d] per out_dtype.
+ */
+int saem_moe_step_host(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const float* logits_host,
+                       const void* x_host, int T, void* out_host, void* stream);
+
+/* Device pointers of the intermediates of the last saem_moe_step (inside the workspace), for
+ * inspection by tests: 0 topk_idx, 1 topk_w, 2 counts, 3 offsets, 4 perm, 5 inv_perm, 6 x_packed,
+ * 7 y_packed, 8 shared_y, 9 h (hidden activations).  NULL for an unknown id. */
+void* saem_step_buffer(saem_ctx* ctx, int which);
+
+/*
+ * Expert cache.  saem_cache_load copies one packed expert (pinned host, saem_slot_bytes) into a
+ * slot with cudaMemcpyAsync on copy_stream and records a completion event; the residency map
+ * changes at once on the host.  slot: 0..slots_per_layer-1 of `layer`, which must be empty
+ * (SLOT_BUSY otherwise: evict first), or SAEM_TEMP: take the next temporary slot round-robin,
+ * dropping whatever it held; a temporary binding serves saem_expert_ffn but is not part of the
+ * residency map.  The copy is ordered after the last FFN that read the slot.  Loading an expert
+ * that already has a fixed slot returns INVALID_ARG.
+ * saem_cache_evict frees the expert's slot (fixed or temporary) on the host table; NOT_RESIDENT
+ * if it has none.  No device work is enqueued.
+ * saem_cache_query: *slot = global slot index, -1 if none; *ready = 1 once the load has completed.
+ * saem_cache_wait: makes consumer_stream wait for the expert's load event (NOT_RESIDENT if none).
+ */
+int saem_cache_load(saem_ctx* ctx, int layer, int expert, int slot, const void* pinned_packed_expert,
+                    void* copy_stream);
+int saem_cache_evict(saem_ctx* ctx, int layer, int expert);
+int saem_cache_query(saem_ctx* ctx, int layer, int expert, int* slot, int* ready);
+int saem_cache_wait(saem_ctx* ctx, int layer, int expert, void* consumer_stream);
+
+/* Reads and clears the sticky device status word (synchronises the device). */
+int saem_last_device_status(saem_ctx* ctx, int* code);
+
+/* Number of kernels this library has launched through `ctx` since creation (host counter). */
+long long saem_launch_count(saem_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAEM_H_ */

@@ -1,0 +1,479 @@
+// Grouped SwiGLU expert FFN over the repacked segments (Sec. IV-E: one dense batched execution
+// per expert over its contiguous rows; Sec. IV-C: weights live in fixed HBM cache slots),
+// written for sm_100a as a weight-streaming kernel:
+//
+//   * Operands are swapped: a 128-row tile of the expert's WEIGHTS is the MMA's M operand and the
+//     segment's tokens are the narrow N operand (16..256), so decode-sized segments still fill the
+//     tensor core's M dimension and every weight byte is read from HBM exactly once per token tile.
+//   * Weight tiles are stored in the slot pre-swizzled (see saem_pack_expert_host), so one
+//     cp.async.bulk per stage lands a 16/32 KB tile in shared memory ready for tcgen05.mma;
+//     activation tiles come through a TMA tensor map with the same 128-byte swizzle.
+//   * One persistent CTA per SM.  The flat list of (expert, token tile, weight-row block,
+//     k-chunk) units of the ACTIVE experts only is cut into equal contiguous ranges, one per CTA
+//     (inactive experts' weights are never touched).  A (expert, token tile, row block) item whose
+//     k-range is split across CTAs is finished by whichever contributor arrives last, which adds
+//     the partial tiles in ascending CTA order -- deterministic, and no CTA ever waits for another.
+//   * Warp roles: warp 0 issues the copies, warp 1 issues tcgen05.mma into TMEM accumulators
+//     (double-buffered when they fit), warps 2..5 read TMEM back (tcgen05.ld), apply SiLU*up or
+//     store y.  Stages are handed over with mbarriers; every wait is bounded and, when it runs out,
+//     sets SAEM_ERR_TIMEOUT in the device status word and makes the CTA drain and return.
+//
+// Two launches per FFN: gate/up (+SiLU*mul -> h, bf16) and down (-> y_packed, fp32).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "saem_internal.h"
+
+namespace saem {
+
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr int kDynSmemMax = 220 * 1024;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+// ------------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit runs out or
+// another role of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    unsigned long long t0 = 0;
+    for (uint32_t i = 0;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u) {
+            if (*abort_flag) return false;
+            unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(status, SAEM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 bytes apart,
+// 8-row groups 1024 bytes apart (the layout both the packed weight tiles and the TMA boxes have).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t idesc_bf16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+}
+
+// --------------------------------------------------------------------------------------- the plan
+struct Plan {
+    int n_active;
+    int total_items;
+    int e[SAEM_MAX_EXPERTS];
+    int slot[SAEM_MAX_EXPERTS];
+    int row0[SAEM_MAX_EXPERTS];
+    int rows[SAEM_MAX_EXPERTS];
+    int item_base[SAEM_MAX_EXPERTS + 1];
+};
+
+struct Item {
+    int a, nb, rb;          // active-expert index, token tile, weight-row block
+    int kc_begin, kc_end;   // this CTA's part of the item's k-chunks
+    int row_start, rows_here, n_eff;
+    long long it;           // global item index
+};
+
+struct ItemWalker {
+    const Plan* plan;
+    long long c, c1;        // next chunk, end of this CTA's range
+    int KC, RB, n_tile;
+    int a_cursor;
+    __device__ __forceinline__ ItemWalker(const Plan* p, long long c0_, long long c1_, int KC_, int RB_, int nt)
+        : plan(p), c(c0_), c1(c1_), KC(KC_), RB(RB_), n_tile(nt), a_cursor(0) {}
+    __device__ __forceinline__ bool next(Item& o) {
+        if (c >= c1) return false;
+        long long it = c / KC;
+        o.it = it;
+        o.kc_begin = (int)(c - it * KC);
+        long long end = (it + 1) * KC;
+        if (end > c1) end = c1;
+        o.kc_end = (int)(end - it * KC);
+        while (a_cursor + 1 < plan->n_active && plan->item_base[a_cursor + 1] <= it) ++a_cursor;
+        o.a = a_cursor;
+        int local = (int)(it - plan->item_base[a_cursor]);
+        o.nb = local / RB;
+        o.rb = local - o.nb * RB;
+        o.row_start = plan->row0[a_cursor] + o.nb * n_tile;
+        int left = plan->rows[a_cursor] - o.nb * n_tile;
+        o.rows_here = left < n_tile ? left : n_tile;
+        o.n_eff = (o.rows_here + 15) & ~15;
+        c = end;
+        return true;
+    }
+};
+
+// ----------------------------------------------------------------------------------------- kernel
+// PHASE 0: h = silu(Wg x) * (Wu x)   (activations = x_packed, reduction over d)
+// PHASE 1: y = Wd h                  (activations = h,        reduction over f)
+template <int PHASE>
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_constant__ CUtensorMap act_map,
+                  int n_stages, int box_rows) {
+    constexpr int W_BYTES = PHASE == 0 ? 2 * kTileBytes : kTileBytes;
+    extern __shared__ uint8_t dyn_smem[];
+    __shared__ Plan plan;
+    __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_flag, last_flag;
+    __shared__ int s_rows[SAEM_MAX_EXPERTS], s_row0[SAEM_MAX_EXPERTS];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int K = PHASE == 0 ? a.d : a.f;
+    const int KC = K / kTileK;
+    const int RB = (PHASE == 0 ? a.f : a.d) / kTileRows;
+    const int n_tile = a.n_tile;
+    const int acc_cols = (PHASE == 0 ? 2 : 1) * n_tile;
+    const int n_acc = (2 * acc_cols <= 512) ? 2 : 1;
+    const uint32_t x_stage_bytes = (uint32_t)n_tile * 128u;
+    const uint32_t stage_bytes = W_BYTES + x_stage_bytes;
+    const uint32_t smem_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+
+    // ---- plan: active experts of this launch, in ascending id ----
+    for (int e = tid; e < a.E; e += kThreads) {
+        int r0 = 0, r1 = a.max_rows;
+        if (a.offsets) { r0 = a.offsets[e]; r1 = a.offsets[e + 1]; }
+        if (r1 > a.max_rows) r1 = a.max_rows;
+        int rows = r1 > r0 ? r1 - r0 : 0;
+        if (!tab.in_subset[e]) rows = 0;
+        if (rows > 0 && tab.slot[e] < 0) {
+            if (blockIdx.x == 0) atomicExch(a.status, SAEM_ERR_NOT_RESIDENT);
+            rows = 0;
+        }
+        s_rows[e] = rows;
+        s_row0[e] = r0;
+    }
+    if (tid == 0) {
+        abort_flag = 0;
+        last_flag = 0;
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_acc_full[s]), 1); mbar_init(smem_u32(&bar_acc_empty[s]), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int n = 0, items = 0;
+        for (int e = 0; e < a.E; ++e) {
+            if (s_rows[e] > 0) {
+                plan.e[n] = e;
+                plan.slot[n] = tab.slot[e];
+                plan.row0[n] = s_row0[e];
+                plan.rows[n] = s_rows[e];
+                plan.item_base[n] = items;
+                items += ((s_rows[e] + n_tile - 1) / n_tile) * RB;
+                ++n;
+            }
+        }
+        plan.item_base[n] = items;
+        plan.n_active = n;
+        plan.total_items = items;
+    }
+    if (warp == 1) {   // TMEM: the whole 512 columns (one CTA per SM)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const long long total_chunks = (long long)plan.total_items * KC;
+    const long long G = gridDim.x;
+    const long long c0 = total_chunks * blockIdx.x / G;
+    const long long c1 = total_chunks * (blockIdx.x + 1) / G;
+    volatile int* abort_p = &abort_flag;
+
+    if (warp == 0) {
+        // =============================== producer ===============================
+        ItemWalker walk(&plan, c0, c1, KC, RB, n_tile);
+        Item it;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        int issued = 0;
+        while (ok && walk.next(it)) {
+            const uint8_t* slot = a.slot_region + (size_t)plan.slot[it.a] * a.slot_bytes;
+            const uint8_t* wbase = slot + (PHASE == 0 ? 0 : (size_t)2 * a.d * a.f * 2) + (size_t)it.rb * KC * W_BYTES;
+            const int n_boxes = (it.rows_here + box_rows - 1) / box_rows;
+            for (int kc = it.kc_begin; kc < it.kc_end; ++kc) {
+                ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, a.status);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t full = smem_u32(&bar_full[stage]);
+                    const uint32_t ws = smem_base + (uint32_t)stage * stage_bytes;
+                    mbar_expect_tx(full, W_BYTES + (uint32_t)(n_boxes * box_rows) * 128u);
+                    const uint8_t* src = wbase + (size_t)kc * W_BYTES;
+                    bulk_g2s(ws, src, kTileBytes, full);
+                    if (PHASE == 0) bulk_g2s(ws + kTileBytes, src + kTileBytes, kTileBytes, full);
+                    for (int b = 0; b < n_boxes; ++b)
+                        tma_2d(ws + W_BYTES + (uint32_t)(b * box_rows) * 128u, &act_map, kc * kTileK,
+                               it.row_start + b * box_rows, full);
+                }
+                ++issued;
+                if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok && issued > 0) {     // let copies already in flight land before the CTA's memory goes away
+            unsigned long long t0 = globaltimer_ns();
+            while (globaltimer_ns() - t0 < 200000ull) {}
+        }
+    } else if (warp == 1) {
+        // =============================== MMA issuer ===============================
+        ItemWalker walk(&plan, c0, c1, KC, RB, n_tile);
+        Item it;
+        int stage = 0, acc = 0;
+        uint32_t phase = 0, acc_phase[2] = {0u, 0u};
+        bool ok = true;
+        while (ok && walk.next(it)) {
+            ok = mbar_wait(smem_u32(&bar_acc_empty[acc]), acc_phase[acc] ^ 1u, abort_p, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * acc_cols);
+            const uint32_t idesc = idesc_bf16(it.n_eff);
+            for (int kc = it.kc_begin; kc < it.kc_end; ++kc) {
+                ok = mbar_wait(smem_u32(&bar_full[stage]), phase, abort_p, a.status);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t ws = smem_base + (uint32_t)stage * stage_bytes;
+                    const uint32_t xs = ws + W_BYTES;
+#pragma unroll
+                    for (int k4 = 0; k4 < kTileK / 16; ++k4) {
+                        const uint32_t accum = (kc > it.kc_begin || k4 > 0) ? 1u : 0u;
+                        const uint64_t bd = smem_desc_sw128(xs + k4 * 32);
+                        tc_mma_bf16(d_tmem, smem_desc_sw128(ws + k4 * 32), bd, idesc, accum);
+                        if (PHASE == 0)
+                            tc_mma_bf16(d_tmem + (uint32_t)n_tile, smem_desc_sw128(ws + kTileBytes + k4 * 32), bd, idesc, accum);
+                    }
+                    tc_commit(smem_u32(&bar_empty[stage]));
+                }
+                __syncwarp();
+                if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            if (lane == 0) tc_commit(smem_u32(&bar_acc_full[acc]));
+            __syncwarp();
+            acc_phase[acc] ^= 1u;
+            if (n_acc == 2) acc ^= 1;
+        }
+    } else {
+        // =============================== epilogue (warps 2..5) ===============================
+        const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int i = q * 32 + lane;            // weight row inside the tile
+        const int epi_tid = tid - 64;
+        ItemWalker walk(&plan, c0, c1, KC, RB, n_tile);
+        Item it;
+        int acc = 0;
+        uint32_t acc_phase[2] = {0u, 0u};
+        bool ok = true;
+        const size_t out_ld = PHASE == 0 ? (size_t)a.f : (size_t)a.d;
+        while (ok && walk.next(it)) {
+            ok = mbar_wait(smem_u32(&bar_acc_full[acc]), acc_phase[acc], abort_p, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            const bool whole = it.kc_begin == 0 && it.kc_end == KC;
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * acc_cols);
+            // which partial slot this CTA's share of the item goes to: it starts inside the item -> 0, else 1
+            const int my_slot = it.kc_begin > 0 ? 0 : 1;
+            float* part = a.partials + ((size_t)blockIdx.x * 2 + my_slot) * a.partial_slot_floats;
+            const size_t col = (size_t)it.rb * kTileRows + i;
+            for (int n0 = 0; n0 < it.n_eff; n0 += 16) {
+                float g[16], u[16];
+                tc_ld16(t_row + (uint32_t)n0, g);
+                if (PHASE == 0) tc_ld16(t_row + (uint32_t)(n_tile + n0), u);
+                if (whole) {
+#pragma unroll
+                    for (int n = 0; n < 16; ++n) {
+                        if (n0 + n < it.rows_here) {
+                            const size_t row = (size_t)(it.row_start + n0 + n);
+                            if (PHASE == 0) {
+                                const float hv = g[n] / (1.f + expf(-g[n])) * u[n];
+                                reinterpret_cast<__nv_bfloat16*>(a.h)[row * out_ld + col] = __float2bfloat16_rn(hv);
+                            } else {
+                                a.y_packed[row * out_ld + col] = g[n];
+                            }
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int n = 0; n < 16; ++n) {
+                        part[(size_t)(n0 + n) * kTileRows + i] = g[n];
+                        if (PHASE == 0) part[(size_t)(n_tile + n0 + n) * kTileRows + i] = u[n];
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[acc]));
+            acc_phase[acc] ^= 1u;
+            if (n_acc == 2) acc ^= 1;
+
+            if (!whole) {
+                // the contributors of this item are the CTAs whose ranges meet [it*KC, (it+1)*KC)
+                const long long s0 = it.it * KC, s1 = s0 + KC - 1;
+                const int b_first = (int)(((s0 + 1) * G - 1) / total_chunks);
+                const int b_last = (int)(((s1 + 1) * G - 1) / total_chunks);
+                const int n_contrib = b_last - b_first + 1;
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (epi_tid == 0) {
+                    int* ctr = a.counters + PHASE * kMaxCtas + b_first;
+                    const int old = atomicAdd(ctr, 1);
+                    const int last = old == n_contrib - 1;
+                    if (last) *ctr = 0;                       // ready for the next launch
+                    last_flag = last;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (last_flag) {
+                    __threadfence();
+                    for (int n = 0; n < it.rows_here; ++n) {
+                        float sg = 0.f, su = 0.f;
+                        for (int b = b_first; b <= b_last; ++b) {       // fixed order: deterministic sum
+                            const float* p = a.partials + ((size_t)b * 2 + (b == b_first ? 1 : 0)) * a.partial_slot_floats;
+                            sg += __ldcg(p + (size_t)n * kTileRows + i);
+                            if (PHASE == 0) su += __ldcg(p + (size_t)(n_tile + n) * kTileRows + i);
+                        }
+                        const size_t row = (size_t)(it.row_start + n);
+                        if (PHASE == 0) {
+                            const float hv = sg / (1.f + expf(-sg)) * su;
+                            reinterpret_cast<__nv_bfloat16*>(a.h)[row * out_ld + col] = __float2bfloat16_rn(hv);
+                        } else {
+                            a.y_packed[row * out_ld + col] = sg;
+                        }
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    }
+}
+
+// ------------------------------------------------------------------------------------------- host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+static bool g_init_done = false;
+
+cudaError_t ffn_tensor_init() {
+    if (g_init_done) return cudaSuccess;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+    g_encode = (EncodeTiledFn)fn;
+    e = cudaFuncSetAttribute(ffn_tensor_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemMax);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(ffn_tensor_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemMax);
+    if (e != cudaSuccess) return e;
+    g_init_done = true;
+    return cudaSuccess;
+}
+
+static bool make_act_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch) {
+    if (!g_init_done) {
+        cudaError_t e = ffn_tensor_init();
+        if (e != cudaSuccess) return e;
+    }
+    const int box_rows = a.n_tile >= 32 ? 32 : 16;
+    alignas(64) CUtensorMap map_x, map_h;
+    if (!make_act_map(&map_x, a.x_packed, a.max_rows, a.d, box_rows)) return cudaErrorInvalidValue;
+    if (!make_act_map(&map_h, a.h, a.max_rows, a.f, box_rows)) return cudaErrorInvalidValue;
+    auto stages_for = [&](int w_bytes) {
+        int sb = w_bytes + a.n_tile * 128;
+        int s = (kDynSmemMax - 1024) / sb;
+        return s > kMaxStages ? kMaxStages : s;
+    };
+    const int s0 = stages_for(2 * kTileBytes), s1 = stages_for(kTileBytes);
+    const size_t smem0 = (size_t)s0 * (2 * kTileBytes + a.n_tile * 128) + 1024;
+    const size_t smem1 = (size_t)s1 * (kTileBytes + a.n_tile * 128) + 1024;
+    ffn_tensor_kernel<0><<<a.n_sm, kThreads, smem0, st>>>(a, tab, map_x, s0, box_rows);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    ffn_tensor_kernel<1><<<a.n_sm, kThreads, smem1, st>>>(a, tab, map_h, s1, box_rows);
+    *n_launch = 2;
+    return cudaGetLastError();
+}
+
+}  // namespace saem

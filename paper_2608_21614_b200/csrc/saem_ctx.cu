@@ -1,0 +1,498 @@
+// Host side of libsaem: context, workspace carving, expert-slot table with asynchronous loads
+// (Sec. IV-C: fixed-size expert cache region, residency map, DMA + event prefetch), the offline
+// weight packer, and the step drivers that chain the four kernels' launchers.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "saem_internal.h"
+
+namespace saem {
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int validate_config(const saem_config* c) {
+    if (!c) return SAEM_ERR_INVALID_ARG;
+    if (c->d_model <= 0 || c->d_ff <= 0 || c->d_model % 128 || c->d_ff % 128) return SAEM_ERR_SHAPE;
+    if (c->n_experts < 1 || c->n_experts > SAEM_MAX_EXPERTS) return SAEM_ERR_SHAPE;
+    if (c->top_k < 1 || c->top_k > c->n_experts) return SAEM_ERR_SHAPE;
+    if (c->max_tokens < 1 || (long long)c->max_tokens * c->top_k > 65535) return SAEM_ERR_SHAPE;
+    if (c->n_layers < 1 || c->slots_per_layer < 0 || c->slots_per_layer > c->n_experts) return SAEM_ERR_SHAPE;
+    if (c->temp_slots < 0 || c->temp_slots > 4096) return SAEM_ERR_SHAPE;
+    if ((long long)c->n_layers * c->slots_per_layer + c->temp_slots < 1) return SAEM_ERR_SHAPE;
+    if (c->out_dtype != SAEM_OUT_F32 && c->out_dtype != SAEM_OUT_BF16) return SAEM_ERR_INVALID_ARG;
+    if (c->ffn_path < SAEM_FFN_AUTO || c->ffn_path > SAEM_FFN_TENSOR) return SAEM_ERR_INVALID_ARG;
+    // repack keeps a [pairs/32][E] table of 16-bit counters in shared memory
+    long long chunks = ((long long)c->max_tokens * c->top_k + 31) / 32;
+    if (chunks * c->n_experts * 2 > 160 * 1024) return SAEM_ERR_UNSUPPORTED;
+    return SAEM_OK;
+}
+
+WorkspaceLayout workspace_layout(const saem_config& c) {
+    WorkspaceLayout L{};
+    const size_t A = 1024;
+    size_t P = (size_t)c.max_tokens * c.top_k, T = c.max_tokens, d = c.d_model, f = c.d_ff, E = c.n_experts;
+    int nt = round_up(c.max_tokens < kMaxNTile ? c.max_tokens : kMaxNTile, 16);
+    L.n_tile_max = nt;
+    L.partial_slot_floats = (size_t)2 * nt * kTileRows;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, A); return o; };
+    L.status = take(256);
+    L.counters = take(sizeof(int) * 2 * kMaxCtas);
+    L.h = take(P * f * 2);
+    L.partials = take((size_t)kMaxCtas * 2 * L.partial_slot_floats * sizeof(float));
+    L.logits = take(T * E * 4);
+    L.x = take(T * d * 2);
+    L.topk_idx = take(P * 4);
+    L.topk_w = take(P * 4);
+    L.counts = take(E * 4);
+    L.offsets = take((E + 1) * 4);
+    L.perm = take(P * 4);
+    L.inv_perm = take(P * 4);
+    L.x_packed = take(P * d * 2);
+    L.y_packed = take(P * d * 4);
+    L.shared_y = take(T * d * 4);
+    L.out = take(T * d * 4);
+    L.total = off;
+    return L;
+}
+
+static int n_tile_for(const saem_ctx* ctx, int max_rows) {
+    int m = max_rows < ctx->cfg.max_tokens ? max_rows : ctx->cfg.max_tokens;   // a token picks an expert once
+    if (m < 1) m = 1;
+    int nt = round_up(m, 16);
+    if (nt > 32) nt = round_up(nt, 32);
+    if (nt > kMaxNTile) nt = kMaxNTile;
+    if (nt > ctx->lay.n_tile_max) nt = ctx->lay.n_tile_max;
+    return nt;
+}
+
+}  // namespace saem
+
+using namespace saem;
+
+#define CUDA_TRY(expr)                                 \
+    do {                                               \
+        cudaError_t e_ = (expr);                       \
+        if (e_ != cudaSuccess) return SAEM_ERR_CUDA;   \
+    } while (0)
+
+extern "C" {
+
+int saem_version(void) { return 100; }
+
+const char* saem_status_string(int s) {
+    switch (s) {
+        case SAEM_OK: return "ok";
+        case SAEM_ERR_INVALID_ARG: return "invalid argument";
+        case SAEM_ERR_SHAPE: return "shape outside the supported range";
+        case SAEM_ERR_ALIGNMENT: return "pointer alignment";
+        case SAEM_ERR_WORKSPACE: return "workspace or slot region too small";
+        case SAEM_ERR_NOT_RESIDENT: return "expert not resident";
+        case SAEM_ERR_SLOT_BUSY: return "slot busy";
+        case SAEM_ERR_TIMEOUT: return "bounded device wait ran out";
+        case SAEM_ERR_CUDA: return "CUDA runtime error";
+        case SAEM_ERR_UNSUPPORTED: return "unsupported configuration";
+    }
+    return "unknown status";
+}
+
+size_t saem_slot_bytes(const saem_config* c) {
+    if (validate_config(c) != SAEM_OK) return 0;
+    return (size_t)3 * c->d_model * c->d_ff * 2;
+}
+
+size_t saem_slot_region_bytes(const saem_config* c) {
+    size_t sb = saem_slot_bytes(c);
+    if (!sb) return 0;
+    return sb * ((size_t)c->n_layers * c->slots_per_layer + c->temp_slots);
+}
+
+size_t saem_workspace_bytes(const saem_config* c) {
+    if (validate_config(c) != SAEM_OK) return 0;
+    return workspace_layout(*c).total;
+}
+
+int saem_create(const saem_config* cfg, void* slot_region, size_t slot_region_bytes, void* ws, size_t ws_bytes,
+                saem_ctx** out) {
+    if (!out) return SAEM_ERR_INVALID_ARG;
+    *out = nullptr;
+    int v = validate_config(cfg);
+    if (v != SAEM_OK) return v;
+    if (!slot_region || !ws) return SAEM_ERR_INVALID_ARG;
+    if (((uintptr_t)slot_region | (uintptr_t)ws) & 1023) return SAEM_ERR_ALIGNMENT;
+    if (slot_region_bytes < saem_slot_region_bytes(cfg)) return SAEM_ERR_WORKSPACE;
+    WorkspaceLayout lay = workspace_layout(*cfg);
+    if (ws_bytes < lay.total) return SAEM_ERR_WORKSPACE;
+
+    saem_ctx* c = new (std::nothrow) saem_ctx();
+    if (!c) return SAEM_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->lay = lay;
+    c->slot_region = (uint8_t*)slot_region;
+    c->slot_bytes = saem_slot_bytes(cfg);
+    c->ws = (uint8_t*)ws;
+    c->n_fixed_slots = cfg->n_layers * cfg->slots_per_layer;
+    c->next_temp = 0;
+    c->launches = 0;
+    c->dynamic_residency = cfg->slots_per_layer < cfg->n_experts || cfg->temp_slots > 0;
+    int n_slots = c->n_fixed_slots + cfg->temp_slots;
+    size_t LE = (size_t)cfg->n_layers * cfg->n_experts;
+    c->slot_of = (int32_t*)malloc(sizeof(int32_t) * LE);
+    c->temp_of = (int32_t*)malloc(sizeof(int32_t) * LE);
+    c->slot_owner = (int32_t*)malloc(sizeof(int32_t) * n_slots);
+    c->ready_ev = (cudaEvent_t*)calloc(n_slots, sizeof(cudaEvent_t));
+    c->ev_pending = (uint8_t*)calloc(n_slots, 1);
+    c->ev_recorded = (uint8_t*)calloc(n_slots, 1);
+    c->read_ev = (cudaEvent_t*)calloc(cfg->n_layers, sizeof(cudaEvent_t));
+    c->read_recorded = (uint8_t*)calloc(cfg->n_layers, 1);
+    c->temp_last_layer = (int32_t*)malloc(sizeof(int32_t) * (cfg->temp_slots > 0 ? cfg->temp_slots : 1));
+    c->pinned_status = nullptr;
+    for (size_t i = 0; i < LE; ++i) c->slot_of[i] = c->temp_of[i] = -1;
+    for (int i = 0; i < n_slots; ++i) c->slot_owner[i] = -1;
+    for (int i = 0; i < cfg->temp_slots; ++i) c->temp_last_layer[i] = -1;
+
+    bool ok = cudaGetDevice(&c->device) == cudaSuccess;
+    ok = ok && cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) == cudaSuccess;
+    if (ok && c->n_sm > kMaxCtas) c->n_sm = kMaxCtas;
+    for (int i = 0; ok && i < n_slots; ++i)
+        ok = cudaEventCreateWithFlags(&c->ready_ev[i], cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < cfg->n_layers; ++i)
+        ok = cudaEventCreateWithFlags(&c->read_ev[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaHostAlloc((void**)&c->pinned_status, sizeof(int), cudaHostAllocDefault) == cudaSuccess;
+    // status word, counters and the step buffers start at zero (h, partials need no clearing)
+    ok = ok && cudaMemsetAsync(c->ws + lay.status, 0, lay.h - lay.status, 0) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(0) == cudaSuccess;
+    if (ok && cfg->ffn_path != SAEM_FFN_SCALAR) ok = ffn_tensor_init() == cudaSuccess;
+    if (!ok) {
+        saem_destroy(c);
+        return SAEM_ERR_CUDA;
+    }
+    *out = c;
+    return SAEM_OK;
+}
+
+void saem_destroy(saem_ctx* c) {
+    if (!c) return;
+    int n_slots = c->n_fixed_slots + c->cfg.temp_slots;
+    if (c->ready_ev)
+        for (int i = 0; i < n_slots; ++i)
+            if (c->ready_ev[i]) cudaEventDestroy(c->ready_ev[i]);
+    if (c->read_ev)
+        for (int i = 0; i < c->cfg.n_layers; ++i)
+            if (c->read_ev[i]) cudaEventDestroy(c->read_ev[i]);
+    if (c->pinned_status) cudaFreeHost(c->pinned_status);
+    free(c->slot_of); free(c->temp_of); free(c->slot_owner); free(c->ready_ev); free(c->ev_pending);
+    free(c->ev_recorded); free(c->read_ev); free(c->read_recorded); free(c->temp_last_layer);
+    delete c;
+}
+
+// ------------------------------------------------------------------------------------ weight packer
+// Tile (rb, kc) of a [rows, K] row-major matrix: 128 rows x 64 elements; row r of the tile is
+// 128 bytes; its 16-byte chunk c lands at chunk position c ^ (r & 7).
+static void pack_matrix(const uint16_t* src, int rows, int K, uint8_t* dst, size_t tile_stride_bytes,
+                        size_t first_tile_offset) {
+    int RB = rows / kTileRows, KC = K / kTileK;
+    for (int rb = 0; rb < RB; ++rb)
+        for (int kc = 0; kc < KC; ++kc) {
+            uint8_t* tile = dst + first_tile_offset + ((size_t)rb * KC + kc) * tile_stride_bytes;
+            for (int r = 0; r < kTileRows; ++r) {
+                const uint16_t* s = src + (size_t)(rb * kTileRows + r) * K + (size_t)kc * kTileK;
+                for (int ch = 0; ch < 8; ++ch)
+                    memcpy(tile + (size_t)r * 128 + (size_t)((ch ^ (r & 7)) * 16), s + ch * 8, 16);
+            }
+        }
+}
+
+int saem_pack_expert_host(const saem_config* cfg, const void* gate, const void* up, const void* down, void* out) {
+    int v = validate_config(cfg);
+    if (v != SAEM_OK) return v;
+    if (!gate || !up || !down || !out) return SAEM_ERR_INVALID_ARG;
+    int d = cfg->d_model, f = cfg->d_ff;
+    uint8_t* o = (uint8_t*)out;
+    // gate/up region: per (f-block, k-chunk) a gate tile followed by the matching up tile
+    pack_matrix((const uint16_t*)gate, f, d, o, 2 * kTileBytes, 0);
+    pack_matrix((const uint16_t*)up, f, d, o, 2 * kTileBytes, kTileBytes);
+    // down region: per (d-block, k-chunk over f) one tile
+    pack_matrix((const uint16_t*)down, d, f, o + (size_t)2 * d * f * 2, kTileBytes, 0);
+    return SAEM_OK;
+}
+
+// ------------------------------------------------------------------------------------------- steps
+static int check_T(saem_ctx* c, int T) {
+    if (!c) return SAEM_ERR_INVALID_ARG;
+    if (T < 0 || T > c->cfg.max_tokens) return SAEM_ERR_SHAPE;
+    return SAEM_OK;
+}
+static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
+int saem_route(saem_ctx* c, const float* logits, int T, int32_t* idx, float* w, void* stream) {
+    int s = check_T(c, T);
+    if (s != SAEM_OK) return s;
+    if (T == 0) return SAEM_OK;
+    if (!logits || !idx || !w) return SAEM_ERR_INVALID_ARG;
+    CUDA_TRY(launch_route(logits, T, c->cfg.n_experts, c->cfg.top_k, c->cfg.renorm, idx, w, (cudaStream_t)stream));
+    c->launches += 1;
+    return SAEM_OK;
+}
+
+int saem_repack(saem_ctx* c, const int32_t* idx, const void* x, int T, int32_t* counts, int32_t* offsets,
+                int32_t* perm, int32_t* inv_perm, void* x_packed, void* stream) {
+    int s = check_T(c, T);
+    if (s != SAEM_OK) return s;
+    if (!counts || !offsets) return SAEM_ERR_INVALID_ARG;
+    if (T > 0 && (!idx || !x || !perm || !inv_perm || !x_packed)) return SAEM_ERR_INVALID_ARG;
+    if (misaligned(x) || misaligned(x_packed)) return SAEM_ERR_ALIGNMENT;
+    int nl = 0;
+    CUDA_TRY(launch_repack(idx, (const uint16_t*)x, T, c->cfg.n_experts, c->cfg.top_k, c->cfg.d_model, counts,
+                           offsets, perm, inv_perm, (uint16_t*)x_packed, (int*)(c->ws + c->lay.status), c->n_sm,
+                           (cudaStream_t)stream, &nl));
+    c->launches += nl;
+    return SAEM_OK;
+}
+
+int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t* offsets, int max_rows,
+                    const int32_t* subset, int n_subset, float* y_packed, void* stream) {
+    if (!c) return SAEM_ERR_INVALID_ARG;
+    const saem_config& g = c->cfg;
+    if (layer < 0 || layer >= g.n_layers) return SAEM_ERR_INVALID_ARG;
+    if (max_rows < 0 || max_rows > g.max_tokens * g.top_k) return SAEM_ERR_SHAPE;
+    if (max_rows == 0) return SAEM_OK;
+    if (!x_packed || !y_packed) return SAEM_ERR_INVALID_ARG;
+    if (!offsets && g.n_experts != 1) return SAEM_ERR_INVALID_ARG;
+    if (misaligned(x_packed) || misaligned(y_packed)) return SAEM_ERR_ALIGNMENT;
+    if (subset && n_subset < 0) return SAEM_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    SlotTable tab;
+    const int32_t* so = c->slot_of + (size_t)layer * g.n_experts;
+    const int32_t* to = c->temp_of + (size_t)layer * g.n_experts;
+    for (int e = 0; e < SAEM_MAX_EXPERTS; ++e) { tab.slot[e] = -1; tab.in_subset[e] = 0; }
+    auto resolve = [&](int e) { return so[e] >= 0 ? so[e] : to[e]; };
+    if (subset) {
+        for (int i = 0; i < n_subset; ++i) {
+            int e = subset[i];
+            if (e < 0 || e >= g.n_experts) return SAEM_ERR_INVALID_ARG;
+            if (resolve(e) < 0) return SAEM_ERR_NOT_RESIDENT;
+        }
+        for (int i = 0; i < n_subset; ++i) { tab.slot[subset[i]] = resolve(subset[i]); tab.in_subset[subset[i]] = 1; }
+    } else {
+        for (int e = 0; e < g.n_experts; ++e) { tab.slot[e] = resolve(e); tab.in_subset[e] = 1; }
+    }
+    // order this stream after loads still in flight for the slots it may read
+    for (int e = 0; e < g.n_experts; ++e) {
+        int s = tab.slot[e];
+        if (s < 0 || !c->ev_pending[s]) continue;
+        cudaError_t q = cudaEventQuery(c->ready_ev[s]);
+        if (q == cudaSuccess) { c->ev_pending[s] = 0; continue; }
+        if (q != cudaErrorNotReady) return SAEM_ERR_CUDA;
+        CUDA_TRY(cudaStreamWaitEvent(st, c->ready_ev[s], 0));
+    }
+
+    FfnArgs a;
+    a.x_packed = (const uint16_t*)x_packed;
+    a.offsets = offsets;
+    a.max_rows = max_rows;
+    a.E = g.n_experts; a.d = g.d_model; a.f = g.d_ff;
+    a.slot_region = c->slot_region;
+    a.slot_bytes = c->slot_bytes;
+    a.h = (uint16_t*)(c->ws + c->lay.h);
+    a.y_packed = y_packed;
+    a.status = (int*)(c->ws + c->lay.status);
+    a.counters = (int*)(c->ws + c->lay.counters);
+    a.partials = (float*)(c->ws + c->lay.partials);
+    a.partial_slot_floats = c->lay.partial_slot_floats;
+    a.n_tile = n_tile_for(c, max_rows);
+    a.n_sm = c->n_sm;
+    int nl = 0;
+    if (g.ffn_path == SAEM_FFN_SCALAR) {
+        CUDA_TRY(launch_ffn_scalar(a, tab, st, &nl));
+    } else {
+        CUDA_TRY(launch_ffn_tensor(a, tab, st, &nl));
+    }
+    c->launches += nl;
+    if (c->dynamic_residency) {
+        CUDA_TRY(cudaEventRecord(c->read_ev[layer], st));
+        c->read_recorded[layer] = 1;
+        for (int e = 0; e < g.n_experts; ++e) {
+            int s = tab.slot[e];
+            if (s >= c->n_fixed_slots) c->temp_last_layer[s - c->n_fixed_slots] = layer;
+        }
+    }
+    return SAEM_OK;
+}
+
+int saem_combine(saem_ctx* c, const float* y, const int32_t* inv_perm, const float* w, int T, const float* shared_y,
+                 void* out, void* stream) {
+    int s = check_T(c, T);
+    if (s != SAEM_OK) return s;
+    if (T == 0) return SAEM_OK;
+    if (!y || !inv_perm || !w || !out) return SAEM_ERR_INVALID_ARG;
+    if (misaligned(y) || misaligned(out) || misaligned(shared_y)) return SAEM_ERR_ALIGNMENT;
+    CUDA_TRY(launch_combine(y, inv_perm, w, T, c->cfg.top_k, c->cfg.d_model, shared_y, out,
+                            c->cfg.out_dtype == SAEM_OUT_BF16, (cudaStream_t)stream));
+    c->launches += 1;
+    return SAEM_OK;
+}
+
+void* saem_step_buffer(saem_ctx* c, int which) {
+    if (!c) return nullptr;
+    const WorkspaceLayout& L = c->lay;
+    size_t offs[10] = {L.topk_idx, L.topk_w, L.counts, L.offsets, L.perm, L.inv_perm, L.x_packed, L.y_packed,
+                       L.shared_y, L.h};
+    if (which < 0 || which >= 10) return nullptr;
+    return c->ws + offs[which];
+}
+
+int saem_moe_step(saem_ctx* c, saem_ctx* sh, int layer, const float* logits, const void* x, int T, void* out,
+                  void* stream) {
+    int s = check_T(c, T);
+    if (s != SAEM_OK) return s;
+    if (T == 0) return SAEM_OK;
+    if (!logits || !x || !out) return SAEM_ERR_INVALID_ARG;
+    const saem_config& g = c->cfg;
+    if (sh && (sh->cfg.n_experts != 1 || sh->cfg.top_k != 1 || sh->cfg.d_model != g.d_model ||
+               sh->cfg.max_tokens < T || layer >= sh->cfg.n_layers))
+        return SAEM_ERR_INVALID_ARG;
+    uint8_t* w = c->ws;
+    const WorkspaceLayout& L = c->lay;
+    int32_t* idx = (int32_t*)(w + L.topk_idx);
+    float* tw = (float*)(w + L.topk_w);
+    int32_t* offsets = (int32_t*)(w + L.offsets);
+    int32_t* inv = (int32_t*)(w + L.inv_perm);
+    float* y = (float*)(w + L.y_packed);
+    float* shy = (float*)(w + L.shared_y);
+    if ((s = saem_route(c, logits, T, idx, tw, stream)) != SAEM_OK) return s;
+    if ((s = saem_repack(c, idx, x, T, (int32_t*)(w + L.counts), offsets, (int32_t*)(w + L.perm), inv,
+                         w + L.x_packed, stream)) != SAEM_OK) return s;
+    if ((s = saem_expert_ffn(c, layer, w + L.x_packed, offsets, T * g.top_k, nullptr, 0, y, stream)) != SAEM_OK)
+        return s;
+    if (sh && (s = saem_expert_ffn(sh, layer, x, nullptr, T, nullptr, 0, shy, stream)) != SAEM_OK) return s;
+    return saem_combine(c, y, inv, tw, T, sh ? shy : nullptr, out, stream);
+}
+
+int saem_moe_step_host(saem_ctx* c, saem_ctx* sh, int layer, const float* logits_h, const void* x_h, int T,
+                       void* out_h, void* stream) {
+    int s = check_T(c, T);
+    if (s != SAEM_OK) return s;
+    if (T == 0) return SAEM_OK;
+    if (!logits_h || !x_h || !out_h) return SAEM_ERR_INVALID_ARG;
+    const saem_config& g = c->cfg;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t* w = c->ws;
+    const WorkspaceLayout& L = c->lay;
+    size_t out_bytes = (size_t)T * g.d_model * (g.out_dtype == SAEM_OUT_BF16 ? 2 : 4);
+    CUDA_TRY(cudaMemcpyAsync(w + L.logits, logits_h, (size_t)T * g.n_experts * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(w + L.x, x_h, (size_t)T * g.d_model * 2, cudaMemcpyHostToDevice, st));
+    s = saem_moe_step(c, sh, layer, (const float*)(w + L.logits), w + L.x, T, w + L.out, stream);
+    if (s != SAEM_OK) return s;
+    CUDA_TRY(cudaMemcpyAsync(out_h, w + L.out, out_bytes, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return SAEM_OK;
+}
+
+// ------------------------------------------------------------------------------------------- cache
+static int check_le(saem_ctx* c, int layer, int expert) {
+    if (!c) return SAEM_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->cfg.n_layers || expert < 0 || expert >= c->cfg.n_experts) return SAEM_ERR_INVALID_ARG;
+    return SAEM_OK;
+}
+
+int saem_cache_load(saem_ctx* c, int layer, int expert, int slot, const void* pinned, void* copy_stream) {
+    int s = check_le(c, layer, expert);
+    if (s != SAEM_OK) return s;
+    if (!pinned) return SAEM_ERR_INVALID_ARG;
+    const saem_config& g = c->cfg;
+    size_t le = (size_t)layer * g.n_experts + expert;
+    cudaStream_t cs = (cudaStream_t)copy_stream;
+    int gslot;
+    int wait_layer = -1;
+    if (slot == SAEM_TEMP) {
+        if (g.temp_slots < 1) return SAEM_ERR_INVALID_ARG;
+        if (c->slot_of[le] >= 0) return SAEM_ERR_INVALID_ARG;
+        int t = c->next_temp;
+        c->next_temp = (t + 1) % g.temp_slots;
+        gslot = c->n_fixed_slots + t;
+        if (c->slot_owner[gslot] >= 0) c->temp_of[c->slot_owner[gslot]] = -1;   // drop the old binding
+        if (c->temp_of[le] >= 0) c->slot_owner[c->temp_of[le]] = -1;             // expert re-bound: free its old temp slot
+        wait_layer = c->temp_last_layer[t];
+        c->temp_of[le] = gslot;
+    } else {
+        if (slot < 0 || slot >= g.slots_per_layer) return SAEM_ERR_INVALID_ARG;
+        if (c->slot_of[le] >= 0) return SAEM_ERR_INVALID_ARG;
+        gslot = layer * g.slots_per_layer + slot;
+        if (c->slot_owner[gslot] >= 0) return SAEM_ERR_SLOT_BUSY;
+        wait_layer = layer;
+        c->slot_of[le] = gslot;
+    }
+    c->slot_owner[gslot] = (int32_t)le;
+    // the copy must not overtake an enqueued FFN that still reads the slot's previous content
+    if (wait_layer >= 0 && c->read_recorded[wait_layer]) {
+        if (cudaStreamWaitEvent(cs, c->read_ev[wait_layer], 0) != cudaSuccess) return SAEM_ERR_CUDA;
+    }
+    if (cudaMemcpyAsync(c->slot_region + (size_t)gslot * c->slot_bytes, pinned, c->slot_bytes, cudaMemcpyHostToDevice,
+                        cs) != cudaSuccess)
+        return SAEM_ERR_CUDA;
+    if (cudaEventRecord(c->ready_ev[gslot], cs) != cudaSuccess) return SAEM_ERR_CUDA;
+    c->ev_pending[gslot] = 1;
+    c->ev_recorded[gslot] = 1;
+    return SAEM_OK;
+}
+
+int saem_cache_evict(saem_ctx* c, int layer, int expert) {
+    int s = check_le(c, layer, expert);
+    if (s != SAEM_OK) return s;
+    size_t le = (size_t)layer * c->cfg.n_experts + expert;
+    if (c->slot_of[le] >= 0) {
+        c->slot_owner[c->slot_of[le]] = -1;
+        c->slot_of[le] = -1;
+        return SAEM_OK;
+    }
+    if (c->temp_of[le] >= 0) {
+        c->slot_owner[c->temp_of[le]] = -1;
+        c->temp_of[le] = -1;
+        return SAEM_OK;
+    }
+    return SAEM_ERR_NOT_RESIDENT;
+}
+
+int saem_cache_query(saem_ctx* c, int layer, int expert, int* slot, int* ready) {
+    int s = check_le(c, layer, expert);
+    if (s != SAEM_OK) return s;
+    size_t le = (size_t)layer * c->cfg.n_experts + expert;
+    int gs = c->slot_of[le] >= 0 ? c->slot_of[le] : c->temp_of[le];
+    if (slot) *slot = gs;
+    if (ready) {
+        *ready = 0;
+        if (gs >= 0 && c->ev_recorded[gs]) {
+            cudaError_t q = cudaEventQuery(c->ready_ev[gs]);
+            if (q == cudaSuccess) { *ready = 1; c->ev_pending[gs] = 0; }
+            else if (q != cudaErrorNotReady) return SAEM_ERR_CUDA;
+        }
+    }
+    return SAEM_OK;
+}
+
+int saem_cache_wait(saem_ctx* c, int layer, int expert, void* consumer) {
+    int s = check_le(c, layer, expert);
+    if (s != SAEM_OK) return s;
+    size_t le = (size_t)layer * c->cfg.n_experts + expert;
+    int gs = c->slot_of[le] >= 0 ? c->slot_of[le] : c->temp_of[le];
+    if (gs < 0 || !c->ev_recorded[gs]) return SAEM_ERR_NOT_RESIDENT;
+    CUDA_TRY(cudaStreamWaitEvent((cudaStream_t)consumer, c->ready_ev[gs], 0));
+    return SAEM_OK;
+}
+
+int saem_last_device_status(saem_ctx* c, int* code) {
+    if (!c || !code) return SAEM_ERR_INVALID_ARG;
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(c->pinned_status, c->ws + c->lay.status, sizeof(int), cudaMemcpyDeviceToHost));
+    *code = *c->pinned_status;
+    CUDA_TRY(cudaMemset(c->ws + c->lay.status, 0, sizeof(int)));
+    return SAEM_OK;
+}
+
+long long saem_launch_count(saem_ctx* c) { return c ? c->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,100 @@
+// Internal declarations shared by the translation units of libsaem (host context + kernels).
+#ifndef SAEM_INTERNAL_H_
+#define SAEM_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "saem.h"
+
+namespace saem {
+
+constexpr int kTileRows = 128;              // weight rows per tile (the MMA M)
+constexpr int kTileK = 64;                  // reduction elements per tile (128 bytes of bf16)
+constexpr int kTileBytes = kTileRows * kTileK * 2;   // 16 KB
+constexpr int kMaxCtas = 160;               // upper bound of the persistent grid (B200: 148 SMs)
+constexpr int kMaxNTile = 256;              // widest token tile (the MMA N)
+
+// Slot index per expert for one FFN launch; travels as a kernel parameter so that the residency
+// table never needs a device mirror.  -1: the expert has no slot or is outside the subset.
+struct SlotTable {
+    int32_t slot[SAEM_MAX_EXPERTS];
+    uint8_t in_subset[SAEM_MAX_EXPERTS];    // 0: skip silently (not asked for)
+};
+
+struct WorkspaceLayout {
+    size_t status;        // int32 status word (+ padding)
+    size_t counters;      // int32[2 * kMaxCtas] split-K arrival counters (gate/up, down)
+    size_t h;             // bf16 [max_rows, d_ff]
+    size_t partials;      // fp32 [kMaxCtas][2][2][n_tile_max][128]
+    size_t logits, x, topk_idx, topk_w, counts, offsets, perm, inv_perm, x_packed, y_packed, shared_y, out;
+    size_t total;
+    int n_tile_max;
+    size_t partial_slot_floats;   // floats of one partial slot (2 accumulators)
+};
+
+WorkspaceLayout workspace_layout(const saem_config& c);
+int validate_config(const saem_config* c);
+inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+
+// ---- kernel launchers (each returns a cudaError_t from the launch) ----
+cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
+                         cudaStream_t st);
+// Returns the number of kernels launched (1 or 2) in *n_launch.
+cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, int k, int d, int32_t* counts,
+                          int32_t* offsets, int32_t* perm, int32_t* inv_perm, uint16_t* x_packed, int* status,
+                          int n_sm, cudaStream_t st, int* n_launch);
+cudaError_t launch_combine(const float* y, const int32_t* inv_perm, const float* w, int T, int k, int d,
+                           const float* shared_y, void* out, int out_bf16, cudaStream_t st);
+
+struct FfnArgs {
+    const uint16_t* x_packed;   // [max_rows, d]
+    const int32_t* offsets;     // [E+1] or nullptr (E == 1: one segment [0, max_rows))
+    int max_rows;
+    int E, d, f;
+    const uint8_t* slot_region;
+    size_t slot_bytes;
+    uint16_t* h;                // [max_rows, f] bf16 workspace
+    float* y_packed;            // [max_rows, d]
+    int* status;
+    int* counters;              // [2 * kMaxCtas]
+    float* partials;
+    size_t partial_slot_floats;
+    int n_tile;                 // token tile for this launch (multiple of 16, <= 256)
+    int n_sm;
+};
+cudaError_t launch_ffn_scalar(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
+cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
+// One-time per process: resolves the driver entry point for tensor-map encoding and opts the
+// kernels into large dynamic shared memory.  Returns cudaSuccess or the failing error.
+cudaError_t ffn_tensor_init();
+
+}  // namespace saem
+
+struct saem_ctx {
+    saem_config cfg;
+    int device;
+    int n_sm;
+    uint8_t* slot_region;
+    size_t slot_bytes;
+    uint8_t* ws;
+    saem::WorkspaceLayout lay;
+    int n_fixed_slots;
+    // residency: fixed slot per (layer, expert), -1 none; temp binding per (layer, expert), -1 none
+    int32_t* slot_of;        // [L*E] global slot index
+    int32_t* temp_of;        // [L*E] global slot index of a temporary binding
+    int32_t* slot_owner;     // [n_slots] layer*E + expert, -1 empty
+    cudaEvent_t* ready_ev;   // [n_slots] recorded on the copy stream after a load
+    uint8_t* ev_pending;     // [n_slots] 1: a load was enqueued and no consumer has been ordered after it yet
+    uint8_t* ev_recorded;    // [n_slots]
+    cudaEvent_t* read_ev;    // [L] recorded on the compute stream after each FFN of that layer
+    uint8_t* read_recorded;  // [L]
+    int32_t* temp_last_layer;  // [temp_slots] layer whose FFN may still be reading the slot, -1 none
+    int next_temp;
+    bool dynamic_residency;  // fewer fixed slots than experts, or temporary slots exist: events are kept
+    long long launches;
+    int* pinned_status;      // pinned host int for status read-back
+};
+
+#endif  // SAEM_INTERNAL_H_

@@ -1,0 +1,239 @@
+"""GPU parity: every C-ABI call against the CPU oracle on the same seeded inputs."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_21614_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+SCALAR, TENSOR = 1, 2
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2608_21614_b200 import binding
+    return binding
+
+
+def _g():
+    import gpu_util
+    return gpu_util
+
+
+@pytest.mark.parametrize("path", [SCALAR, TENSOR])
+def test_c1_every_call(oracle, path):
+    g = _g()
+    li = gen.layer_inputs(gen.layer_config("c1"))
+    layer = g.make_layer(li, path)
+    ref, stats = g.run_stepwise_and_compare(layer, li, oracle)
+    # run twice: bit-identical outputs (no atomics decide any order)
+    y1, o1 = layer.y_packed.clone(), layer.out.clone()
+    layer.step(g.dev(li.logits), g.dev(li.x), li.cfg.tokens)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, layer.y_packed) and torch.equal(o1, layer.out)
+    layer.close()
+
+
+@pytest.mark.parametrize("path", [SCALAR, TENSOR])
+@pytest.mark.parametrize("T,E,k,d,f,fs", [
+    (1, 1, 1, 128, 128, 0),          # dense FFN, one token
+    (1, 60, 4, 256, 384, 256),       # decode batch 1: four one-row segments, 56 empty, shared expert
+    (9, 8, 8, 128, 256, 0),          # k == E
+    (33, 60, 4, 256, 128, 0),        # E not a multiple of 32, ragged T
+    (70, 128, 8, 128, 128, 128),     # E = 128, k = 8
+    (300, 8, 2, 256, 256, 0),        # segments beyond one 16..64-row tile; fused repack limit
+    (1500, 16, 2, 128, 128, 0),      # two-kernel repack, several 256-row token tiles per expert
+])
+def test_small_shapes(oracle, path, T, E, k, d, f, fs):
+    g = _g()
+    cfg = gen.LayerConfig("t", d, f, E, k, T, fs, "zipf", 1.1, seed=T + E)
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, path)
+    g.run_stepwise_and_compare(layer, li, oracle)
+    layer.close()
+
+
+@pytest.mark.parametrize("path", [SCALAR, TENSOR])
+def test_segment_sizes_around_tile_edges(oracle, path):
+    """One expert, k = 1: the segment is the whole batch; sizes straddle every tile boundary."""
+    g = _g()
+    d, f = 256, 256
+    rng = np.random.default_rng(77)
+    gate, up, down = gen.expert_weights(rng, d, f)
+    from paper_2608_21614_b200.layer import MoELayer
+    layer = MoELayer(d, f, 1, 1, 300, ffn_path=path)
+    layer.load_all([gate], [up], [down])
+    for T in (1, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257, 300):
+        x = gen.activations(rng, T, d)
+        ref = oracle.expert_ffn(x, np.array([0, T], np.int32), [gate], [up], [down])
+        y = torch.full((300, d), float("nan"), dtype=torch.float32, device="cuda:0")
+        import paper_2608_21614_b200.binding as B
+        B.saem_expert_ffn(layer.ctx.handle, 0, g.dev(x), None, T, None, y)
+        torch.cuda.synchronize()
+        g.assert_close(g.host(y[:T]), ref, "T=%d" % T)
+        assert torch.isnan(y[T:]).all(), "rows beyond the segment were written (T=%d)" % T
+    assert layer.device_status() == 0
+    layer.close()
+
+
+def test_route_special_values(oracle, B):
+    g = _g()
+    rows = [
+        [-0.0, 0.0, -np.inf, np.nan, 1.0, -1.0, 0.5, 0.5],
+        [np.inf, 1.0, np.inf, 0.0, 0.0, 0.0, 0.0, 0.0],
+        [-np.inf] * 8,
+        [0.0] * 8,
+        [300.0, 0.0, -300.0, 1.0, 2.0, 3.0, 4.0, 5.0],
+        [np.nan] * 8,
+    ]
+    logits = np.array(rows, np.float32)
+    rng = np.random.default_rng(1)
+    quant = rng.integers(-2, 3, size=(64, 8)).astype(np.float32)          # many exact ties
+    logits = np.concatenate([logits, quant])
+    for k, renorm in ((1, 1), (3, 1), (8, 1), (3, 0)):
+        cfg = B.make_config(128, 128, 8, k, len(logits), renorm=renorm)
+        ctx = B.Context(cfg)
+        idx = torch.empty((len(logits), k), dtype=torch.int32, device="cuda:0")
+        w = torch.empty((len(logits), k), dtype=torch.float32, device="cuda:0")
+        B.saem_route(ctx.handle, g.dev(logits), len(logits), idx, w)
+        torch.cuda.synchronize()
+        ridx, rw = oracle.route(logits, k, renorm=bool(renorm))
+        assert np.array_equal(g.host(idx), ridx), (k, renorm)
+        assert np.isfinite(g.host(w)).all()
+        assert np.abs(g.host(w).astype(np.float64) - rw).max() <= g.W_TOL, (k, renorm)
+        ctx.close()
+
+
+@pytest.mark.parametrize("E,k", [(8, 2), (60, 4), (64, 6), (128, 8), (128, 128), (33, 33)])
+def test_route_random(oracle, B, E, k):
+    g = _g()
+    rng = np.random.default_rng(E * 7 + k)
+    T = 257
+    logits = rng.standard_normal((T, E)).astype(np.float32) * 3
+    ctx = B.Context(B.make_config(128, 128, E, k, T))
+    idx = torch.empty((T, k), dtype=torch.int32, device="cuda:0")
+    w = torch.empty((T, k), dtype=torch.float32, device="cuda:0")
+    B.saem_route(ctx.handle, g.dev(logits), T, idx, w)
+    ridx, rw = oracle.route(logits, k)
+    assert np.array_equal(g.host(idx), ridx)
+    assert np.abs(g.host(w).astype(np.float64) - rw).max() <= g.W_TOL
+    ctx.close()
+
+
+def test_repack_skew_and_paper_example(oracle, B):
+    g = _g()
+    # the paper's worked example (Sec. IV-E)
+    idx = np.array([[0, 2], [1, 2], [1, 3], [0, 2]], np.int32)
+    cases = [(idx, 4)]
+    cases.append((np.full((50, 1), 3, np.int32), 6))                      # every token picks the same expert
+    rng = np.random.default_rng(2)
+    cases.append((np.stack([rng.permutation(60)[:4] for _ in range(777)]).astype(np.int32), 60))
+    cases.append((np.stack([rng.permutation(64)[:6] for _ in range(2048)]).astype(np.int32), 64))   # prefill size
+    for idx, E in cases:
+        T, k = idx.shape
+        d = 128
+        x = rng.integers(0, 65535, size=(T, d)).astype(np.uint16)
+        ctx = B.Context(B.make_config(d, 128, E, k, T))
+        P = T * k
+        counts = torch.empty(E, dtype=torch.int32, device="cuda:0")
+        offsets = torch.empty(E + 1, dtype=torch.int32, device="cuda:0")
+        perm = torch.empty(P, dtype=torch.int32, device="cuda:0")
+        inv = torch.empty(P, dtype=torch.int32, device="cuda:0")
+        xp = torch.empty((P, d), dtype=torch.uint16, device="cuda:0")
+        B.saem_repack(ctx.handle, g.dev(idx), g.dev(x), T, counts, offsets, perm, inv, xp)
+        rc, ro, rp, ri, rx = oracle.repack(idx, x, E)
+        assert np.array_equal(g.host(counts), rc)
+        assert np.array_equal(g.host(offsets), ro)
+        assert np.array_equal(g.host(perm), rp)
+        assert np.array_equal(g.host(inv), ri)
+        assert np.array_equal(g.host(xp), rx)
+        assert B.saem_last_device_status(ctx.handle) == 0
+        ctx.close()
+
+
+def test_step_calls_agree_bit_for_bit(oracle):
+    """saem_moe_step and saem_moe_step_host give the bits of the four separate calls."""
+    g = _g()
+    cfg = gen.LayerConfig("t", 256, 384, 12, 3, 20, 256, "zipf", 1.1, seed=5)
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, TENSOR)
+    logits, x = g.dev(li.logits), g.dev(li.x)
+    ref_out = layer.step(logits, x, cfg.tokens).clone()
+    out2 = torch.empty_like(ref_out)
+    layer.step_fused_call(logits, x, cfg.tokens, out2)
+    torch.cuda.synchronize()
+    assert torch.equal(ref_out, out2)
+    lh = torch.from_numpy(li.logits).pin_memory()
+    xh = torch.from_numpy(li.x).pin_memory()
+    oh = torch.empty((cfg.tokens, cfg.d_model), dtype=torch.float32).pin_memory()
+    layer.step_host(lh, xh, cfg.tokens, oh)
+    assert torch.equal(ref_out.cpu(), oh)
+    ref = oracle.moe_step(li.logits, li.x, cfg.top_k, li.gate, li.up, li.down, shared=li.shared)
+    g.assert_close(oh.numpy(), ref["out"], "out via host call")
+    layer.close()
+
+
+def test_bf16_output_option(oracle):
+    g = _g()
+    from paper_2608_21614_b200 import binding as B
+    cfg = gen.layer_config("c1")
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, TENSOR, out_dtype=B.SAEM_OUT_BF16)
+    out = layer.step(g.dev(li.logits), g.dev(li.x), cfg.tokens)
+    torch.cuda.synchronize()
+    ref = oracle.moe_step(li.logits, li.x, cfg.top_k, li.gate, li.up, li.down)
+    g.assert_close(gen.bf16_bits_to_f32(g.host(out)), ref["out"], "bf16 out")
+    layer.close()
+
+
+def test_error_statuses(B):
+    g = _g()
+    cfg = B.make_config(128, 128, 4, 2, 8)
+    ctx = B.Context(cfg)
+    z = torch.zeros(4096, dtype=torch.float32, device="cuda:0")
+    zi = torch.zeros(4096, dtype=torch.int32, device="cuda:0")
+    assert B.saem_route(ctx.handle, z, 9, zi, z, check=False) == B.SAEM_ERR_SHAPE          # T = max_tokens + 1
+    assert B.saem_route(ctx.handle, z, 8, zi, z, check=False) == B.SAEM_OK                 # T = max_tokens
+    assert B.saem_route(ctx.handle, None, 8, zi, z, check=False) == B.SAEM_ERR_INVALID_ARG
+    assert B.saem_expert_ffn(ctx.handle, 1, z, zi, 4, None, z, check=False) == B.SAEM_ERR_INVALID_ARG   # bad layer
+    assert B.saem_expert_ffn(ctx.handle, 0, z, zi, 17, None, z, check=False) == B.SAEM_ERR_SHAPE
+    assert B.saem_expert_ffn(ctx.handle, 0, z, zi, 4, [2], z, check=False) == B.SAEM_ERR_NOT_RESIDENT
+    assert B.saem_cache_evict(ctx.handle, 0, 1, check=False) == B.SAEM_ERR_NOT_RESIDENT
+    assert B.saem_cache_load(ctx.handle, 0, 1, 9, z, check=False) == B.SAEM_ERR_INVALID_ARG              # bad slot
+    assert B.saem_cache_load(ctx.handle, 0, 1, B.SAEM_TEMP, z, check=False) == B.SAEM_ERR_INVALID_ARG    # no temp slots
+    assert B.saem_cache_query(ctx.handle, 0, 1) == (-1, 0)
+    bad = B.make_config(100, 128, 4, 2, 8)
+    assert B.saem_slot_bytes(bad) == 0
+    assert B.saem_create_status(bad, ctx.slot_ptr, 1 << 30, ctx.ws_ptr, 1 << 30) == B.SAEM_ERR_SHAPE
+    assert B.saem_create_status(cfg, ctx.slot_ptr + 16, 1 << 30, ctx.ws_ptr, 1 << 30) == B.SAEM_ERR_ALIGNMENT
+    assert B.saem_create_status(cfg, ctx.slot_ptr, 16, ctx.ws_ptr, 1 << 30) == B.SAEM_ERR_WORKSPACE
+    ctx.close()
+
+
+@pytest.mark.parametrize("path", [SCALAR, TENSOR])
+def test_absent_expert_sets_device_status_and_leaves_rows(oracle, path, B):
+    g = _g()
+    cfg = gen.LayerConfig("t", 128, 128, 4, 2, 16, seed=3)
+    li = gen.layer_inputs(cfg)
+    from paper_2608_21614_b200.layer import MoELayer
+    layer = MoELayer(128, 128, 4, 2, 16, ffn_path=path)
+    for e in (0, 1, 3):                                   # expert 2 never loaded
+        layer.load_expert(0, e, e, li.gate[e], li.up[e], li.down[e])
+    layer.route(g.dev(li.logits), 16)
+    layer.repack(g.dev(li.x), 16)
+    layer.y_packed.fill_(float("nan"))
+    layer.expert_ffn(16)
+    torch.cuda.synchronize()
+    ref = oracle.moe_step(li.logits, li.x, 2, li.gate, li.up, li.down)
+    assert ref["counts"][2] > 0
+    assert layer.device_status() == B.SAEM_ERR_NOT_RESIDENT
+    assert layer.device_status() == 0                      # reading clears it
+    o = ref["offsets"]
+    y = g.host(layer.y_packed)
+    assert np.isnan(y[o[2]:o[3]]).all()
+    keep = np.r_[0:o[2], o[3]:o[4]]
+    g.assert_close(y[keep], ref["y_packed"][keep], "other segments")
+    layer.close()
