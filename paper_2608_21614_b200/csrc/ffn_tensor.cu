@@ -176,7 +176,8 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     __shared__ Plan plan;
     __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_flag, last_flag;
+    __shared__ int abort_flag, last_flag, s_ncontrib;
+    __shared__ short s_contrib[256];            // contributors of a split item (at most K/64 <= 256)
     __shared__ int s_rows[SAEM_MAX_EXPERTS], s_row0[SAEM_MAX_EXPERTS];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -370,15 +371,21 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
             if (n_acc == 2) acc ^= 1;
 
             if (!whole) {
-                // the contributors of this item are the CTAs whose ranges meet [it*KC, (it+1)*KC)
+                // The contributors of this item are the CTAs whose (non-empty) ranges meet
+                // [it*KC, (it+1)*KC).  CTA b owns chunks [b*total/G, (b+1)*total/G); when there are
+                // fewer chunks than CTAs some ranges are empty, so the list is walked, not counted.
                 const long long s0 = it.it * KC, s1 = s0 + KC - 1;
-                const int b_first = (int)(((s0 + 1) * G - 1) / total_chunks);
-                const int b_last = (int)(((s1 + 1) * G - 1) / total_chunks);
-                const int n_contrib = b_last - b_first + 1;
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (epi_tid == 0) {
-                    int* ctr = a.counters + PHASE * kMaxCtas + b_first;
+                    int n_contrib = 0;
+                    for (long long c = s0; c <= s1;) {
+                        const int b = (int)(((c + 1) * G - 1) / total_chunks);    // the CTA that owns chunk c
+                        s_contrib[n_contrib++] = (short)b;
+                        c = ((long long)(b + 1) * total_chunks) / G;              // first chunk of the next CTA
+                    }
+                    s_ncontrib = n_contrib;
+                    int* ctr = a.counters + PHASE * kMaxCtas + s_contrib[0];
                     const int old = atomicAdd(ctr, 1);
                     const int last = old == n_contrib - 1;
                     if (last) *ctr = 0;                       // ready for the next launch
@@ -389,8 +396,9 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                     __threadfence();
                     for (int n = 0; n < it.rows_here; ++n) {
                         float sg = 0.f, su = 0.f;
-                        for (int b = b_first; b <= b_last; ++b) {       // fixed order: deterministic sum
-                            const float* p = a.partials + ((size_t)b * 2 + (b == b_first ? 1 : 0)) * a.partial_slot_floats;
+                        for (int ci = 0; ci < s_ncontrib; ++ci) {       // fixed order: deterministic sum
+                            const int b = s_contrib[ci];
+                            const float* p = a.partials + ((size_t)b * 2 + (ci == 0 ? 1 : 0)) * a.partial_slot_floats;
                             sg += __ldcg(p + (size_t)n * kTileRows + i);
                             if (PHASE == 0) su += __ldcg(p + (size_t)(n_tile + n) * kTileRows + i);
                         }

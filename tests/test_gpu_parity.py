@@ -23,7 +23,7 @@ def _g():
     return gpu_util
 
 
-@pytest.mark.parametrize("path", [SCALAR, TENSOR])
+@pytest.mark.parametrize("path", [SCALAR, TENSOR], ids=["scalar", "tensor"])
 def test_c1_every_call(oracle, path):
     g = _g()
     li = gen.layer_inputs(gen.layer_config("c1"))
@@ -37,7 +37,7 @@ def test_c1_every_call(oracle, path):
     layer.close()
 
 
-@pytest.mark.parametrize("path", [SCALAR, TENSOR])
+@pytest.mark.parametrize("path", [SCALAR, TENSOR], ids=["scalar", "tensor"])
 @pytest.mark.parametrize("T,E,k,d,f,fs", [
     (1, 1, 1, 128, 128, 0),          # dense FFN, one token
     (1, 60, 4, 256, 384, 256),       # decode batch 1: four one-row segments, 56 empty, shared expert
@@ -56,7 +56,7 @@ def test_small_shapes(oracle, path, T, E, k, d, f, fs):
     layer.close()
 
 
-@pytest.mark.parametrize("path", [SCALAR, TENSOR])
+@pytest.mark.parametrize("path", [SCALAR, TENSOR], ids=["scalar", "tensor"])
 def test_segment_sizes_around_tile_edges(oracle, path):
     """One expert, k = 1: the segment is the whole batch; sizes straddle every tile boundary."""
     g = _g()
@@ -111,7 +111,7 @@ def test_route_special_values(oracle, B):
 def test_route_random(oracle, B, E, k):
     g = _g()
     rng = np.random.default_rng(E * 7 + k)
-    T = 257
+    T = 257 if k <= 8 else 40          # the repack table bounds pairs x experts
     logits = rng.standard_normal((T, E)).astype(np.float32) * 3
     ctx = B.Context(B.make_config(128, 128, E, k, T))
     idx = torch.empty((T, k), dtype=torch.int32, device="cuda:0")
@@ -213,7 +213,7 @@ def test_error_statuses(B):
     ctx.close()
 
 
-@pytest.mark.parametrize("path", [SCALAR, TENSOR])
+@pytest.mark.parametrize("path", [SCALAR, TENSOR], ids=["scalar", "tensor"])
 def test_absent_expert_sets_device_status_and_leaves_rows(oracle, path, B):
     g = _g()
     cfg = gen.LayerConfig("t", 128, 128, 4, 2, 16, seed=3)
