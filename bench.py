@@ -35,9 +35,9 @@ WORKLOADS = {
     "c4": "c4: Qwen-MoE-shaped layer, d_model=2048, 60 experts top-4 + shared d_ff=5632, routed d_ff=1408",
 }
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of the two FFN kernels of one step, from the ncu
-# capture summarised in profiles/ (None until a capture of this exact configuration exists)
-NCU_FFN_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of the two FFN kernels of one step of workload c2
+# with all 8 experts active, from the ncu capture summarised in profiles/ffn_tensor_c2_decode.md
+NCU_FFN_TRAFFIC_BYTES = {"c2": 2836640000}
 
 
 def measured_peaks():
@@ -62,7 +62,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
 
@@ -194,7 +194,7 @@ def run_ours(args):
                        "l2": "layer weights %.2f GB vs 126 MB L2: inputs larger than L2, no flush" % weight_gb,
                        "distinct_weight_sets": args.distinct, "replicas": world},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_FFN_TRAFFIC_BYTES, "peak_source": which,
+                         "traffic": NCU_FFN_TRAFFIC_BYTES.get(args.workload) if (args.tokens is None and n_active == E) else None, "peak_source": which,
                          "kernel": "saem_expert_ffn (gate/up + down kernels%s)" % (", routed + shared calls" if cfg.d_ff_shared else ""),
                          "algorithmic_bytes": ffn_bytes, "avg_ms": ffn_avg_ms,
                          "frac_of_nominal_8000": achieved / 8000.0},
@@ -264,7 +264,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--distinct", type=int, default=8, help="distinct expert weight sets to generate (1..8)")
