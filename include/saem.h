@@ -206,6 +206,36 @@ int saem_cache_evict(saem_ctx* ctx, int layer, int expert);
 int saem_cache_query(saem_ctx* ctx, int layer, int expert, int* slot, int* ready);
 int saem_cache_wait(saem_ctx* ctx, int layer, int expert, void* consumer_stream);
 
+/*
+ * (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
+ *
+ * saem_expert_ffn_static is saem_expert_ffn for code that must not, or cannot, call cudaMalloc: a
+ * plugin inside an application that owns the whole memory pool, a latency-critical loop where an
+ * allocation may block, a process whose pool is already exhausted.  It needs no saem_ctx and no
+ * workspace: the hidden activations h[max_rows, d_ff] (bf16) live in a fixed array inside the
+ * library, SAEM_STATIC_SCRATCH_ELEMS elements (2 MiB) that every GPU which loads the library
+ * holds until the process exits.  The function calls no allocating routine of any kind.
+ *
+ *   x_packed[max_rows, d_model] bf16, offsets[n_experts + 1] int32, y_packed[max_rows, d_model] fp32:
+ *   device, caller-owned, 16-byte aligned, with the meaning they have in saem_expert_ffn.
+ *   packed_experts: device, n_experts packed experts (saem_pack_expert_host layout) back to back,
+ *   expert e at byte offset e * 3 * d_model * d_ff * 2 -- for instance the slots of one layer of a
+ *   fully resident slot region.  Plain scalar kernels; results agree with saem_expert_ffn within
+ *   its tolerance.
+ *
+ * Limits and errors: max_rows * d_ff > SAEM_STATIC_SCRATCH_ELEMS returns SAEM_ERR_WORKSPACE and
+ * enqueues nothing; shapes and alignment as for saem_expert_ffn (SAEM_ERR_SHAPE, _ALIGNMENT,
+ * _INVALID_ARG).  The first call on a device looks the array's device address up (a short
+ * host-side set-up with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents: every
+ * element a call reads it has written itself first, so nothing needs clearing, but two calls
+ * whose kernels may overlap on the GPU (different streams, no ordering between them) race on it
+ * -- order them on one stream or with events.
+ */
+enum { SAEM_STATIC_SCRATCH_ELEMS = 1 << 20 };
+int saem_expert_ffn_static(const void* x_packed, const int32_t* offsets, int n_experts, int max_rows,
+                           int d_model, int d_ff, const void* packed_experts, float* y_packed, void* stream);
+
 /* Reads and clears the sticky device status word (synchronises the device). */
 int saem_last_device_status(saem_ctx* ctx, int* code);
 

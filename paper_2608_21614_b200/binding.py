@@ -65,6 +65,7 @@ def _load() -> C.CDLL:
         "saem_cache_wait": (i32, [vp, i32, i32, vp]),
         "saem_last_device_status": (i32, [vp, C.POINTER(i32)]),
         "saem_launch_count": (C.c_longlong, [vp]),
+        "saem_expert_ffn_static": (i32, [vp, vp, i32, i32, i32, i32, vp, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -77,7 +78,7 @@ _lib = _load()
 EXPORTS = ("saem_version saem_status_string saem_slot_bytes saem_slot_region_bytes saem_workspace_bytes "
            "saem_create saem_destroy saem_pack_expert_host saem_route saem_repack saem_expert_ffn saem_combine "
            "saem_moe_step saem_moe_step_host saem_step_buffer saem_cache_load saem_cache_evict saem_cache_query "
-           "saem_cache_wait saem_last_device_status saem_launch_count").split()
+           "saem_cache_wait saem_last_device_status saem_launch_count saem_expert_ffn_static").split()
 
 
 def library_path() -> str:
@@ -247,6 +248,21 @@ def saem_last_device_status(ctx) -> int:
 
 def saem_launch_count(ctx) -> int:
     return int(_lib.saem_launch_count(ctx))
+
+
+SAEM_STATIC_SCRATCH_ELEMS = 1 << 20
+
+
+def saem_expert_ffn_static(x_packed, offsets, n_experts, max_rows, d_model, d_ff, packed_experts, y_packed,
+                           stream=None, check=True) -> int:
+    """The expert FFN for callers that cannot allocate device memory: no context, no workspace;
+    the hidden activations use a fixed 2 MiB array inside the library (max_rows * d_ff elements at
+    most SAEM_STATIC_SCRATCH_ELEMS).  Calls that may overlap on the GPU race on that array."""
+    code = _lib.saem_expert_ffn_static(_ptr(x_packed), _ptr(offsets), n_experts, max_rows, d_model, d_ff,
+                                       _ptr(packed_experts), _ptr(y_packed), _stream(stream))
+    if check:
+        _check(code, "saem_expert_ffn_static")
+    return code
 
 
 # ------------------------------------------------------------------------- memory plumbing (torch)
