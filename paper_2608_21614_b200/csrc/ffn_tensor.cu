@@ -30,6 +30,7 @@ constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
 constexpr int kDynSmemMax = 220 * 1024;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr long long kSplitBelowItemsPerCta = 6;   // split items across CTAs only below this many items per CTA
 
 // ------------------------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -239,10 +240,15 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
+    // Decode-sized work (few items per CTA) is cut at k-chunk granularity so that every SM streams
+    // the same number of bytes; with many items per CTA whole items are dealt out instead and no
+    // partial tiles are needed.
     const long long total_chunks = (long long)plan.total_items * KC;
     const long long G = gridDim.x;
-    const long long c0 = total_chunks * blockIdx.x / G;
-    const long long c1 = total_chunks * (blockIdx.x + 1) / G;
+    const bool split_k = (long long)plan.total_items < kSplitBelowItemsPerCta * G;
+    const long long c0 = split_k ? total_chunks * blockIdx.x / G : ((long long)plan.total_items * blockIdx.x / G) * KC;
+    const long long c1 = split_k ? total_chunks * (blockIdx.x + 1) / G
+                                 : ((long long)plan.total_items * (blockIdx.x + 1) / G) * KC;
     volatile int* abort_p = &abort_flag;
 
     if (warp == 0) {
@@ -394,20 +400,40 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (last_flag) {
                     __threadfence();
-                    for (int n = 0; n < it.rows_here; ++n) {
-                        float sg = 0.f, su = 0.f;
-                        for (int ci = 0; ci < s_ncontrib; ++ci) {       // fixed order: deterministic sum
-                            const int b = s_contrib[ci];
-                            const float* p = a.partials + ((size_t)b * 2 + (ci == 0 ? 1 : 0)) * a.partial_slot_floats;
-                            sg += __ldcg(p + (size_t)n * kTileRows + i);
-                            if (PHASE == 0) su += __ldcg(p + (size_t)(n_tile + n) * kTileRows + i);
+                    // eight token columns at a time: 8 (16 with the up half) independent L2 loads
+                    // in flight per thread and contributor; contributors added in ascending order
+                    const int nc = s_ncontrib;
+                    for (int n0 = 0; n0 < it.rows_here; n0 += 8) {
+                        float sg[8], su[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) sg[j] = su[j] = 0.f;
+                        for (int ci = 0; ci < nc; ++ci) {
+                            const float* p = a.partials + ((size_t)s_contrib[ci] * 2 + (ci == 0 ? 1 : 0)) * a.partial_slot_floats +
+                                             (size_t)n0 * kTileRows + i;
+                            float vg[8], vu[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) vg[j] = __ldcg(p + (size_t)j * kTileRows);
+                            if (PHASE == 0) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) vu[j] = __ldcg(p + (size_t)(n_tile + j) * kTileRows);
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                sg[j] += vg[j];
+                                if (PHASE == 0) su[j] += vu[j];
+                            }
                         }
-                        const size_t row = (size_t)(it.row_start + n);
-                        if (PHASE == 0) {
-                            const float hv = sg / (1.f + expf(-sg)) * su;
-                            reinterpret_cast<__nv_bfloat16*>(a.h)[row * out_ld + col] = __float2bfloat16_rn(hv);
-                        } else {
-                            a.y_packed[row * out_ld + col] = sg;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (n0 + j < it.rows_here) {
+                                const size_t row = (size_t)(it.row_start + n0 + j);
+                                if (PHASE == 0) {
+                                    const float hv = sg[j] / (1.f + expf(-sg[j])) * su[j];
+                                    reinterpret_cast<__nv_bfloat16*>(a.h)[row * out_ld + col] = __float2bfloat16_rn(hv);
+                                } else {
+                                    a.y_packed[row * out_ld + col] = sg[j];
+                                }
+                            }
                         }
                     }
                 }

@@ -160,17 +160,20 @@ class StageTrace:
     rankings: np.ndarray
     zipf_s: float
     seed: int
-    reshuffled: int
+    reshuffled: float
 
     def stage_of(self, step: int) -> int:
         return int(np.searchsorted(self.boundaries, step, side="right") - 1)
 
 
 def stage_trace(n_steps: int, n_layers: int, n_experts: int, zipf_s: float, seed: int,
-                mean_stage_len: float = 200.0, reshuffled: Optional[int] = 2) -> StageTrace:
+                mean_stage_len: float = 200.0, reshuffled: Optional[float] = 3.2) -> StageTrace:
     """Stage lengths iid Geometric(1/mean) until n_steps; per layer, stage 0 has a uniform
     random ranking and every later stage re-draws the ranks of ``reshuffled`` randomly chosen
-    experts among themselves (``None``: an independent fresh ranking per stage)."""
+    experts among themselves (a fractional value m + p means m or m + 1 experts with probability
+    1 - p and p; ``None``: an independent fresh ranking per stage).  The default 3.2 gives a
+    measured adjacent-stage coherence (Eq. 1 of the paper) of about 0.89 for 8 experts, top-2,
+    Zipf exponent 1.2 -- the paper's reported mean."""
     st = _streams(seed)
     lens = []
     while sum(lens) < n_steps:
@@ -186,10 +189,11 @@ def stage_trace(n_steps: int, n_layers: int, n_experts: int, zipf_s: float, seed
                 rk[s, l] = st["rank"].permutation(n_experts) + 1
             else:
                 cur = rk[s - 1, l].copy()
-                pos = st["rank"].choice(n_experts, size=min(reshuffled, n_experts), replace=False)
+                m = int(np.floor(reshuffled)) + int(st["rank"].random() < (reshuffled - np.floor(reshuffled)))
+                pos = st["rank"].choice(n_experts, size=min(m, n_experts), replace=False)
                 cur[pos] = cur[st["rank"].permutation(pos)]
                 rk[s, l] = cur
-    return StageTrace(n_steps, bounds, rk, zipf_s, seed, -1 if reshuffled is None else reshuffled)
+    return StageTrace(n_steps, bounds, rk, zipf_s, seed, -1.0 if reshuffled is None else float(reshuffled))
 
 
 def trace_logits(trace: StageTrace, step: int, layer: int, batch: int) -> np.ndarray:

@@ -1,0 +1,192 @@
+"""Expert-slot cache on the GPU: load / evict / query / wait semantics, ordering of loads against
+enqueued FFNs, and the partially resident stack (50 % of the experts per layer in fixed slots,
+misses through temporary slots, planner at stage boundaries) against full residency and against
+an independent host simulation of the same policy."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_21614_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+
+def _small_experts(n, d, f, seed):
+    rng = np.random.default_rng(seed)
+    return [gen.expert_weights(rng, d, f) for _ in range(n)]
+
+
+def test_cache_api_semantics():
+    import gpu_util as g
+    from paper_2608_21614_b200 import binding as B
+    d, f, E = 128, 128, 4
+    ws = _small_experts(E, d, f, 1)
+    cfg = B.make_config(d, f, E, 2, 8, n_layers=2, slots_per_layer=2, temp_slots=2)
+    ctx = B.Context(cfg)
+    h = ctx.handle
+    packed = [ctx.pack(*w) for w in ws]
+    cs = torch.cuda.Stream()
+    assert B.saem_cache_query(h, 0, 0) == (-1, 0)
+    B.saem_cache_load(h, 0, 0, 0, packed[0], cs)
+    slot, _ = B.saem_cache_query(h, 0, 0)
+    assert slot == 0
+    cs.synchronize()
+    assert B.saem_cache_query(h, 0, 0) == (0, 1)
+    assert B.saem_cache_load(h, 0, 1, 0, packed[1], cs, check=False) == B.SAEM_ERR_SLOT_BUSY
+    assert B.saem_cache_load(h, 0, 0, 1, packed[0], cs, check=False) == B.SAEM_ERR_INVALID_ARG      # already resident
+    B.saem_cache_load(h, 1, 3, 1, packed[3], cs)                       # layer 1, slot 1 -> global slot 3
+    assert B.saem_cache_query(h, 1, 3)[0] == 3
+    # temporary slots: round-robin over the pool (global slots 4, 5), old bindings dropped
+    B.saem_cache_load(h, 0, 2, B.SAEM_TEMP, packed[2], cs)
+    B.saem_cache_load(h, 1, 0, B.SAEM_TEMP, packed[0], cs)
+    assert B.saem_cache_query(h, 0, 2)[0] == 4 and B.saem_cache_query(h, 1, 0)[0] == 5
+    B.saem_cache_load(h, 1, 1, B.SAEM_TEMP, packed[1], cs)             # recycles pool slot 0
+    assert B.saem_cache_query(h, 0, 2)[0] == -1 and B.saem_cache_query(h, 1, 1)[0] == 4
+    assert B.saem_cache_load(h, 0, 0, B.SAEM_TEMP, packed[0], cs, check=False) == B.SAEM_ERR_INVALID_ARG
+    B.saem_cache_evict(h, 0, 0)
+    assert B.saem_cache_query(h, 0, 0) == (-1, 0)
+    assert B.saem_cache_evict(h, 0, 0, check=False) == B.SAEM_ERR_NOT_RESIDENT
+    assert B.saem_cache_wait(h, 0, 0, None, check=False) == B.SAEM_ERR_NOT_RESIDENT
+    assert B.saem_cache_wait(h, 1, 3, None, check=False) == B.SAEM_OK
+    torch.cuda.synchronize()
+    ctx.close()
+
+
+def test_load_is_ordered_after_enqueued_reads_and_before_later_ones(oracle):
+    """Swap the expert in a slot right after enqueuing an FFN that reads it: the first result
+    uses the old weights, the next one the new weights."""
+    import gpu_util as g
+    from paper_2608_21614_b200 import binding as B
+    d, f, T = 256, 256, 24
+    wa, wb = _small_experts(2, d, f, 5)
+    cfg = B.make_config(d, f, 2, 1, T, slots_per_layer=1, temp_slots=1)
+    ctx = B.Context(cfg)
+    h = ctx.handle
+    pa, pb = ctx.pack(*wa), ctx.pack(*wb)
+    cs = torch.cuda.Stream()
+    rng = np.random.default_rng(2)
+    x = gen.activations(rng, T, d)
+    xd = g.dev(x)
+    off0 = g.dev(np.array([0, T, T], np.int32))          # every row belongs to expert 0
+    off1 = g.dev(np.array([0, 0, T], np.int32))          # ... to expert 1
+    y0 = torch.zeros((T, d), dtype=torch.float32, device="cuda:0")
+    y1 = torch.zeros((T, d), dtype=torch.float32, device="cuda:0")
+    B.saem_cache_load(h, 0, 0, 0, pa, cs)
+    for _ in range(3):                                     # a queue of reads of the slot
+        B.saem_expert_ffn(h, 0, xd, off0, T, [0], y0)
+    B.saem_cache_evict(h, 0, 0)
+    B.saem_cache_load(h, 0, 1, 0, pb, cs)                  # same slot, other expert, no host sync in between
+    assert B.saem_expert_ffn(h, 0, xd, off0, T, [0], y0, check=False) == B.SAEM_ERR_NOT_RESIDENT
+    B.saem_expert_ffn(h, 0, xd, off1, T, [1], y1)
+    torch.cuda.synchronize()
+    seg = np.array([0, T], np.int32)
+    g.assert_close(g.host(y0), oracle.expert_ffn(x, seg, [wa[0]], [wa[1]], [wa[2]]), "old expert")
+    g.assert_close(g.host(y1), oracle.expert_ffn(x, seg, [wb[0]], [wb[1]], [wb[2]]), "new expert")
+    assert B.saem_last_device_status(h) == 0
+    ctx.close()
+
+
+def _run_stack(trace, weights, L, E, k, d, f, C, temp, batch, steps, keep):
+    from paper_2608_21614_b200.stack import StackRunner
+    run = StackRunner(d, f, E, k, L, C, temp, batch, weights)
+    # warm set: the C most popular experts of stage 0 (stand-in for the calibration warm-up)
+    run.warm([list(np.argsort(trace.rankings[0, l])[:C]) for l in range(L)])
+    outs = []
+    bounds = set(int(b) for b in trace.boundaries[1:])
+    for t in range(steps):
+        if t in bounds:
+            run.boundary()
+        lg = np.stack([gen.trace_logits(trace, t, l, batch) for l in range(L)])
+        x = gen.trace_activations(trace, t, batch, d)
+        out = run.step(torch.from_numpy(lg).cuda(), torch.from_numpy(x).cuda())
+        if t in keep:
+            torch.cuda.synchronize()
+            outs.append(out.clone())
+    torch.cuda.synchronize()
+    assert __import__("paper_2608_21614_b200.binding", fromlist=["x"]).saem_last_device_status(run.h) == 0
+    stats = run.stats
+    final = [list(s) for s in run.slot_expert]
+    store = run.store
+    return outs, stats, final, run
+
+
+def _simulate(trace, oracle, L, E, k, C, temp, batch, steps):
+    """Independent host simulation of the policy: residency sets, a ring of temporary slots,
+    the pairwise-swap planner at boundaries; routing from the oracle."""
+    res = [set(int(e) for e in np.argsort(trace.rankings[0, l])[:C]) for l in range(L)]
+    ring = [None] * temp
+    nxt = 0
+    log = np.zeros((L, E), np.int64)
+    st = dict(active=0, hits=0, temp_hits=0, demand=0, boundary=0, pair_total=0, pair_hits=0)
+    bounds = set(int(b) for b in trace.boundaries[1:])
+    for t in range(steps):
+        if t in bounds:
+            for l in range(L):
+                while True:
+                    non = [e for e in range(E) if e not in res[l]]
+                    best = min(non, key=lambda e: (-log[l, e], e))
+                    worst = min(res[l], key=lambda e: (log[l, e], -e))
+                    if log[l, best] <= log[l, worst]:
+                        break
+                    res[l].remove(worst)
+                    res[l].add(best)
+                    st["boundary"] += 1
+                    ring = [None if r == (l, best) else r for r in ring]
+            log[:] = 0
+        for l in range(L):
+            idx, _ = oracle.route(gen.trace_logits(trace, t, l, batch), k)
+            cnt = np.bincount(idx.ravel(), minlength=E)
+            need = []
+            for e in np.nonzero(cnt)[0]:
+                e = int(e)
+                st["active"] += 1
+                st["pair_total"] += int(cnt[e])
+                if e in res[l]:
+                    st["hits"] += 1
+                    st["pair_hits"] += int(cnt[e])
+                else:
+                    need.append(e)
+                    if (l, e) in ring:
+                        st["temp_hits"] += 1
+            while True:
+                missing = [e for e in need if (l, e) not in ring]
+                if not missing:
+                    break
+                for e in missing:
+                    ring[nxt] = (l, e)
+                    nxt = (nxt + 1) % temp
+                    st["demand"] += 1
+            log[l] += cnt
+    return st, [sorted(r) for r in res]
+
+
+def test_half_resident_stack_equals_full_residency_and_simulation(oracle):
+    import gpu_util as g
+    L, E, k, d, f, batch, steps = 3, 8, 2, 256, 256, 4, 40
+    trace = gen.stage_trace(steps, L, E, 1.2, seed=11, mean_stage_len=8.0)
+    assert len(trace.boundaries) >= 3
+    weights = _small_experts(6, d, f, 3)                     # 24 (layer, expert) pairs share 6 weight sets
+    keep = set(range(steps))
+    full, st_full, _, run_full = _run_stack(trace, weights, L, E, k, d, f, E, 0, batch, steps, keep)
+    half, st_half, final_half, run_half = _run_stack(trace, weights, L, E, k, d, f, E // 2, 4, batch, steps, keep)
+    # routing does not depend on placement: identical bits under 50 % and 100 % residency
+    for a, b in zip(full, half):
+        assert torch.equal(a, b)
+    assert st_full.chr() == 1.0 and st_full.demand_loads == 0 and st_full.boundary_loads == 0
+    # the policy bookkeeping equals an independent simulation, number for number
+    sim, sim_final = _simulate(trace, oracle, L, E, k, E // 2, 4, batch, steps)
+    assert (st_half.active, st_half.hits, st_half.temp_hits) == (sim["active"], sim["hits"], sim["temp_hits"])
+    assert (st_half.pair_total, st_half.pair_hits) == (sim["pair_total"], sim["pair_hits"])
+    assert st_half.demand_loads == sim["demand"] and st_half.boundary_loads == sim["boundary"]
+    assert [sorted(s) for s in final_half] == sim_final
+    assert 0.3 < st_half.chr() < 1.0 and st_half.demand_loads > 0 and st_half.boundary_loads > 0
+    # floating-point parity of sampled layer-steps against the oracle (same weight mapping)
+    for t in (0, int(trace.boundaries[1]), steps - 1):
+        x = gen.trace_activations(trace, t, batch, d)
+        for l in range(L):
+            ws = [run_half.store.weights(l, e) for e in range(E)]
+            ref = oracle.moe_step(gen.trace_logits(trace, t, l, batch), x, k, [w[0] for w in ws],
+                                  [w[1] for w in ws], [w[2] for w in ws])
+            g.assert_close(g.host(half[t][l]), ref["out"], "step %d layer %d" % (t, l))
+    run_full.close()
+    run_half.close()
