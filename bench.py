@@ -93,6 +93,23 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(values, device):
+    """Element-wise maximum of `values` over all ranks (identity when not distributed): the
+    time of a multi-replica run is the slowest replica's."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def aggregate_tokens_per_s(world, tokens_per_step, steps, slowest_ms):
+    """Whole-job throughput of `world` independent replicas timed by the slowest one."""
+    return world * tokens_per_step * steps / (slowest_ms * 1e-3)
+
+
 def build_inputs(args):
     from paper_2608_21614_b200 import inputs as gen
     cfg = gen.layer_config(args.workload, tokens=args.tokens, routing=args.routing)
@@ -174,19 +191,14 @@ def run_ours(args):
         layer.step_host(lh, xh, T, oh)
     e2e_s = time.perf_counter() - t0
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_s / Ke], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_step_s = float(t[0]), float(t[1])
-    else:
-        e2e_step_s = e2e_s / Ke
+    total_ms, e2e_step_s = max_over_ranks([total_ms, e2e_s / Ke], device)
     if rank == 0:
         peaks, which = measured_peaks()
         ffn_avg_ms = sum(ffn_ms) / len(ffn_ms)
         achieved = ffn_bytes / (ffn_avg_ms * 1e-3) / 1e9
         peak = float(peaks["hbm_gbs"])
         line = {
-            "metric": METRIC, "value": world * T * K / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": aggregate_tokens_per_s(world, T, K, total_ms), "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / K, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOADS[args.workload], "tokens_per_step": T, "active_experts": n_active,

@@ -12,6 +12,8 @@ namespace saem {
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ inv_perm, const float* __restrict__ w,
                int T, int k, int d, const float* __restrict__ shared_y, void* __restrict__ out, int out_bf16) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int vec_per_row = d >> 2;
     const long long total = (long long)T * vec_per_row;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
@@ -49,8 +51,8 @@ cudaError_t launch_combine(const float* y, const int32_t* inv_perm, const float*
     long long total = (long long)T * (d / 4);
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    combine_kernel<<<(int)blocks, 256, 0, st>>>(y, inv_perm, w, T, k, d, shared_y, out, out_bf16);
-    return cudaGetLastError();
+    return launch_pdl(combine_kernel, dim3((unsigned)blocks), dim3(256), 0, st, y, inv_perm, w, T, k, d, shared_y, out,
+                      out_bf16);
 }
 
 }  // namespace saem

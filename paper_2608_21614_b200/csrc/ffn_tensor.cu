@@ -26,7 +26,9 @@
 
 namespace saem {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                 // warp 0 copies, warp 1 MMA, warps 2..9 epilogue
+constexpr int kEpiThreads = 256;
+constexpr int kGateUpMaxTile = 128;           // widest token tile of the gate/up phase (two accumulator sets fit TMEM)
 constexpr int kMaxStages = 8;
 constexpr int kDynSmemMax = 220 * 1024;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
@@ -169,7 +171,7 @@ struct ItemWalker {
 // PHASE 0: h = silu(Wg x) * (Wu x)   (activations = x_packed, reduction over d)
 // PHASE 1: y = Wd h                  (activations = h,        reduction over f)
 template <int PHASE>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_constant__ CUtensorMap act_map,
                   int n_stages, int box_rows) {
     constexpr int W_BYTES = PHASE == 0 ? 2 * kTileBytes : kTileBytes;
@@ -179,7 +181,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag, last_flag, s_ncontrib;
     __shared__ short s_contrib[256];            // contributors of a split item (at most K/64 <= 256)
-    __shared__ int s_rows[SAEM_MAX_EXPERTS], s_row0[SAEM_MAX_EXPERTS];
+    __shared__ int s_warp_act[kThreads / 32], s_warp_items[kThreads / 32];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int K = PHASE == 0 ? a.d : a.f;
@@ -188,56 +190,77 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     const int n_tile = a.n_tile;
     const int acc_cols = (PHASE == 0 ? 2 : 1) * n_tile;
     const int n_acc = (2 * acc_cols <= 512) ? 2 : 1;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < n_acc * acc_cols) tmem_cols <<= 1;
     const uint32_t x_stage_bytes = (uint32_t)n_tile * 128u;
     const uint32_t stage_bytes = W_BYTES + x_stage_bytes;
     const uint32_t smem_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
 
-    // ---- plan: active experts of this launch, in ascending id ----
-    for (int e = tid; e < a.E; e += kThreads) {
-        int r0 = 0, r1 = a.max_rows;
-        if (a.offsets) { r0 = a.offsets[e]; r1 = a.offsets[e + 1]; }
-        if (r1 > a.max_rows) r1 = a.max_rows;
-        int rows = r1 > r0 ? r1 - r0 : 0;
-        if (!tab.in_subset[e]) rows = 0;
-        if (rows > 0 && tab.slot[e] < 0) {
-            if (blockIdx.x == 0) atomicExch(a.status, SAEM_ERR_NOT_RESIDENT);
-            rows = 0;
-        }
-        s_rows[e] = rows;
-        s_row0[e] = r0;
-    }
+    // ---- set-up that does not depend on earlier kernels: barriers, tensor memory ----
     if (tid == 0) {
         abort_flag = 0;
         last_flag = 0;
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_acc_full[s]), 1); mbar_init(smem_u32(&bar_acc_empty[s]), 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_acc_full[s]), 1); mbar_init(smem_u32(&bar_acc_empty[s]), kEpiThreads / 32); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
-    if (tid == 0) {
-        int n = 0, items = 0;
-        for (int e = 0; e < a.E; ++e) {
-            if (s_rows[e] > 0) {
-                plan.e[n] = e;
-                plan.slot[n] = tab.slot[e];
-                plan.row0[n] = s_row0[e];
-                plan.rows[n] = s_rows[e];
-                plan.item_base[n] = items;
-                items += ((s_rows[e] + n_tile - 1) / n_tile) * RB;
-                ++n;
-            }
-        }
-        plan.item_base[n] = items;
-        plan.n_active = n;
-        plan.total_items = items;
-    }
-    if (warp == 1) {   // TMEM: the whole 512 columns (one CTA per SM)
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512));
+    if (warp == 1) {   // TMEM: only the columns this launch needs, so that two CTAs can share an SM
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(tmem_cols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
+    // Everything below reads what the preceding kernels of the stream wrote (offsets, x_packed, h).
+    // Under programmatic dependent launch this kernel may have started before they finished.
+    pdl_wait();
+    pdl_launch_dependents();
+
+    // ---- plan: active experts of this launch, in ascending id (one thread per expert) ----
+    {
+        const int e = tid;
+        int rows = 0, r0 = 0;
+        if (e < a.E) {
+            int r1 = a.max_rows;
+            if (a.offsets) { r0 = a.offsets[e]; r1 = a.offsets[e + 1]; }
+            if (r1 > a.max_rows) r1 = a.max_rows;
+            rows = r1 > r0 ? r1 - r0 : 0;
+            if (!tab.in_subset[e]) rows = 0;
+            if (rows > 0 && tab.slot[e] < 0) {
+                if (blockIdx.x == 0) atomicExch(a.status, SAEM_ERR_NOT_RESIDENT);
+                rows = 0;
+            }
+        }
+        const int my_items = rows > 0 ? ((rows + n_tile - 1) / n_tile) * RB : 0;
+        int act_inc = rows > 0 ? 1 : 0, item_inc = my_items;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int na = __shfl_up_sync(0xffffffffu, act_inc, o), ni = __shfl_up_sync(0xffffffffu, item_inc, o);
+            if (lane >= o) { act_inc += na; item_inc += ni; }
+        }
+        if (lane == 31) { s_warp_act[warp] = act_inc; s_warp_items[warp] = item_inc; }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        int base_act = 0, base_items = 0, tot_act = 0, tot_items = 0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) {
+            if (w < warp) { base_act += s_warp_act[w]; base_items += s_warp_items[w]; }
+            tot_act += s_warp_act[w];
+            tot_items += s_warp_items[w];
+        }
+        if (rows > 0) {
+            const int n = base_act + act_inc - 1;
+            plan.e[n] = e;
+            plan.slot[n] = tab.slot[e];
+            plan.row0[n] = r0;
+            plan.rows[n] = rows;
+            plan.item_base[n] = base_items + item_inc - my_items;
+        }
+        if (tid == 0) {
+            plan.item_base[tot_act] = tot_items;
+            plan.n_active = tot_act;
+            plan.total_items = tot_items;
+        }
+        __syncthreads();
+    }
     const uint32_t tmem_base = tmem_base_s;
 
     // Decode-sized work (few items per CTA) is cut at k-chunk granularity so that every SM streams
@@ -325,8 +348,10 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
             if (n_acc == 2) acc ^= 1;
         }
     } else {
-        // =============================== epilogue (warps 2..5) ===============================
+        // =============================== epilogue (warps 2..9) ===============================
+        // Two warps per TMEM lane quarter; each takes half of the item's token columns.
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;
         const int i = q * 32 + lane;            // weight row inside the tile
         const int epi_tid = tid - 64;
         ItemWalker walk(&plan, c0, c1, KC, RB, n_tile);
@@ -345,7 +370,9 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
             const int my_slot = it.kc_begin > 0 ? 0 : 1;
             float* part = a.partials + ((size_t)blockIdx.x * 2 + my_slot) * a.partial_slot_floats;
             const size_t col = (size_t)it.rb * kTileRows + i;
-            for (int n0 = 0; n0 < it.n_eff; n0 += 16) {
+            const int split = ((it.n_eff >> 1) + 15) & ~15;
+            const int n_begin = half == 0 ? 0 : split, n_end = half == 0 ? split : it.n_eff;
+            for (int n0 = n_begin; n0 < n_end; n0 += 16) {
                 float g[16], u[16];
                 tc_ld16(t_row + (uint32_t)n0, g);
                 if (PHASE == 0) tc_ld16(t_row + (uint32_t)(n_tile + n0), u);
@@ -355,7 +382,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                         if (n0 + n < it.rows_here) {
                             const size_t row = (size_t)(it.row_start + n0 + n);
                             if (PHASE == 0) {
-                                const float hv = g[n] / (1.f + expf(-g[n])) * u[n];
+                                const float hv = __fdividef(g[n], 1.f + __expf(-g[n])) * u[n];
                                 reinterpret_cast<__nv_bfloat16*>(a.h)[row * out_ld + col] = __float2bfloat16_rn(hv);
                             } else {
                                 a.y_packed[row * out_ld + col] = g[n];
@@ -382,7 +409,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                 // fewer chunks than CTAs some ranges are empty, so the list is walked, not counted.
                 const long long s0 = it.it * KC, s1 = s0 + KC - 1;
                 __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (epi_tid == 0) {
                     int n_contrib = 0;
                     for (long long c = s0; c <= s1;) {
@@ -397,13 +424,14 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                     if (last) *ctr = 0;                       // ready for the next launch
                     last_flag = last;
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (last_flag) {
                     __threadfence();
                     // eight token columns at a time: 8 (16 with the up half) independent L2 loads
                     // in flight per thread and contributor; contributors added in ascending order
                     const int nc = s_ncontrib;
-                    for (int n0 = 0; n0 < it.rows_here; n0 += 8) {
+                    const int r_end = n_end < it.rows_here ? n_end : it.rows_here;
+                    for (int n0 = n_begin; n0 < r_end; n0 += 8) {
                         float sg[8], su[8];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) sg[j] = su[j] = 0.f;
@@ -428,7 +456,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                             if (n0 + j < it.rows_here) {
                                 const size_t row = (size_t)(it.row_start + n0 + j);
                                 if (PHASE == 0) {
-                                    const float hv = sg[j] / (1.f + expf(-sg[j])) * su[j];
+                                    const float hv = __fdividef(sg[j], 1.f + __expf(-sg[j])) * su[j];
                                     reinterpret_cast<__nv_bfloat16*>(a.h)[row * out_ld + col] = __float2bfloat16_rn(hv);
                                 } else {
                                     a.y_packed[row * out_ld + col] = sg[j];
@@ -437,7 +465,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                         }
                     }
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, 256;" ::: "memory");
             }
         }
     }
@@ -447,7 +475,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols));
     }
 }
 
@@ -491,23 +519,33 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
         if (e != cudaSuccess) return e;
     }
     const int box_rows = a.n_tile >= 32 ? 32 : 16;
+    const int nt0 = a.n_tile < kGateUpMaxTile ? a.n_tile : kGateUpMaxTile, nt1 = a.n_tile;
     alignas(64) CUtensorMap map_x, map_h;
     if (!make_act_map(&map_x, a.x_packed, a.max_rows, a.d, box_rows)) return cudaErrorInvalidValue;
     if (!make_act_map(&map_h, a.h, a.max_rows, a.f, box_rows)) return cudaErrorInvalidValue;
-    auto stages_for = [&](int w_bytes) {
-        int sb = w_bytes + a.n_tile * 128;
-        int s = (kDynSmemMax - 1024) / sb;
+    // Small token tiles (decode): two CTAs per SM, each with half the shared memory, so that one
+    // CTA's prologue, epilogue and split-item reduction overlap the other's streaming.
+    const bool two_per_sm = a.n_tile <= 64;
+    const int smem_budget = two_per_sm ? 108 * 1024 : kDynSmemMax;
+    auto stages_for = [&](int w_bytes, int nt) {
+        int sb = w_bytes + nt * 128;
+        int s = (smem_budget - 1024) / sb;
         return s > kMaxStages ? kMaxStages : s;
     };
-    const int s0 = stages_for(2 * kTileBytes), s1 = stages_for(kTileBytes);
-    const size_t smem0 = (size_t)s0 * (2 * kTileBytes + a.n_tile * 128) + 1024;
-    const size_t smem1 = (size_t)s1 * (kTileBytes + a.n_tile * 128) + 1024;
-    ffn_tensor_kernel<0><<<a.n_sm, kThreads, smem0, st>>>(a, tab, map_x, s0, box_rows);
-    cudaError_t e = cudaGetLastError();
+    const int s0 = stages_for(2 * kTileBytes, nt0), s1 = stages_for(kTileBytes, nt1);
+    const size_t smem0 = (size_t)s0 * (2 * kTileBytes + nt0 * 128) + 1024;
+    const size_t smem1 = (size_t)s1 * (kTileBytes + nt1 * 128) + 1024;
+    FfnArgs args0 = a, args1 = a;
+    args0.n_tile = nt0;
+    args1.n_tile = nt1;
+    args0.partial_slot_floats = (size_t)2 * nt0 * kTileRows;
+    args1.partial_slot_floats = (size_t)2 * nt1 * kTileRows;
+    const dim3 grid((unsigned)(two_per_sm ? 2 * a.n_sm : a.n_sm)), block(kThreads);
+    cudaError_t e = launch_pdl(ffn_tensor_kernel<0>, grid, block, smem0, st, args0, tab, map_x, s0, box_rows);
     if (e != cudaSuccess) return e;
-    ffn_tensor_kernel<1><<<a.n_sm, kThreads, smem1, st>>>(a, tab, map_h, s1, box_rows);
+    e = launch_pdl(ffn_tensor_kernel<1>, grid, block, smem1, st, args1, tab, map_h, s1, box_rows);
     *n_launch = 2;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace saem

@@ -101,6 +101,8 @@ repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict_
                     int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ perm,
                     int32_t* __restrict__ inv_perm, uint16_t* __restrict__ x_packed, int* __restrict__ status) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
+    pdl_wait();
+    pdl_launch_dependents();
     const int P = T * k, n_chunks = (P + 31) >> 5;
     RepackSmem& sm = *reinterpret_cast<RepackSmem*>(smem_raw);
     uint16_t* table = reinterpret_cast<uint16_t*>(smem_raw + sizeof(RepackSmem));
@@ -123,6 +125,8 @@ repack_index_kernel(const int32_t* __restrict__ idx, int T, int E, int k, int32_
                     int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
                     int* __restrict__ status) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
+    pdl_wait();
+    pdl_launch_dependents();
     const int P = T * k, n_chunks = (P + 31) >> 5;
     RepackSmem& sm = *reinterpret_cast<RepackSmem*>(smem_raw);
     uint16_t* table = reinterpret_cast<uint16_t*>(smem_raw + sizeof(RepackSmem));
@@ -133,6 +137,8 @@ repack_index_kernel(const int32_t* __restrict__ idx, int T, int E, int k, int32_
 __global__ void __launch_bounds__(256)
 repack_gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm,
                      const int32_t* __restrict__ offsets, int E, int k, int d, uint16_t* __restrict__ x_packed) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int total = offsets[E];
     const int sub = threadIdx.x >> 6, nsub = blockDim.x >> 6;     // 64 threads per row
     for (int r = blockIdx.x * nsub + sub; r < total; r += gridDim.x * nsub) {
@@ -160,18 +166,16 @@ cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, i
         int grid = (P + rows_per_cta - 1) / rows_per_cta;
         if (grid < 1) grid = 1;
         if (grid > n_sm) grid = n_sm;
-        repack_fused_kernel<<<grid, kRepackThreads, smem, st>>>(idx, x, T, E, k, d, counts, offsets, perm, inv_perm,
-                                                                x_packed, status);
         *n_launch = 1;
-        return cudaGetLastError();
+        return launch_pdl(repack_fused_kernel, dim3(grid), dim3(kRepackThreads), smem, st, idx, x, T, E, k, d, counts,
+                          offsets, perm, inv_perm, x_packed, status);
     }
     size_t smem = base + (size_t)n_chunks * 32;
-    repack_index_kernel<<<1, 1024, smem, st>>>(idx, T, E, k, counts, offsets, perm, inv_perm, status);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(repack_index_kernel, dim3(1), dim3(1024), smem, st, idx, T, E, k, counts, offsets, perm,
+                               inv_perm, status);
     if (e != cudaSuccess) return e;
-    repack_gather_kernel<<<n_sm * 4, 256, 0, st>>>(x, perm, offsets, E, k, d, x_packed);
     *n_launch = 2;
-    return cudaGetLastError();
+    return launch_pdl(repack_gather_kernel, dim3(n_sm * 4), dim3(256), 0, st, x, perm, offsets, E, k, d, x_packed);
 }
 
 }  // namespace saem

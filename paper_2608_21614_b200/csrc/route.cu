@@ -28,6 +28,8 @@ __device__ __forceinline__ float key_value(uint32_t k) {
 __global__ void __launch_bounds__(kRouteWarps * 32)
 route_kernel(const float* __restrict__ logits, int T, int E, int k, int renorm, int32_t* __restrict__ idx,
              float* __restrict__ w) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * kRouteWarps + (threadIdx.x >> 5);
     if (t >= T) return;
@@ -110,8 +112,7 @@ route_kernel(const float* __restrict__ logits, int T, int E, int k, int renorm, 
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
                          cudaStream_t st) {
     int blocks = (T + kRouteWarps - 1) / kRouteWarps;
-    route_kernel<<<blocks, kRouteWarps * 32, 0, st>>>(logits, T, E, k, renorm, idx, w);
-    return cudaGetLastError();
+    return launch_pdl(route_kernel, dim3(blocks), dim3(kRouteWarps * 32), 0, st, logits, T, E, k, renorm, idx, w);
 }
 
 }  // namespace saem

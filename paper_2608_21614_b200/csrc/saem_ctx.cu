@@ -41,7 +41,11 @@ WorkspaceLayout workspace_layout(const saem_config& c) {
     L.status = take(256);
     L.counters = take(sizeof(int) * 2 * kMaxCtas);
     L.h = take(P * f * 2);
-    L.partials = take((size_t)kMaxCtas * 2 * L.partial_slot_floats * sizeof(float));
+    {   // split-K partial tiles: the larger of the two launch shapes (see launch_ffn_tensor)
+        size_t small_tile = (size_t)2 * (nt < 64 ? nt : 64) * kTileRows;
+        size_t a = (size_t)kMaxCtas * 2 * small_tile, b = (size_t)kMaxSms * 2 * L.partial_slot_floats;
+        L.partials = take((a > b ? a : b) * sizeof(float));
+    }
     L.logits = take(T * E * 4);
     L.x = take(T * d * 2);
     L.topk_idx = take(P * 4);
@@ -155,7 +159,7 @@ int saem_create(const saem_config* cfg, void* slot_region, size_t slot_region_by
 
     bool ok = cudaGetDevice(&c->device) == cudaSuccess;
     ok = ok && cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device) == cudaSuccess;
-    if (ok && c->n_sm > kMaxCtas) c->n_sm = kMaxCtas;
+    if (ok && c->n_sm > kMaxSms) c->n_sm = kMaxSms;
     for (int i = 0; ok && i < n_slots; ++i)
         ok = cudaEventCreateWithFlags(&c->ready_ev[i], cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; ok && i < cfg->n_layers; ++i)

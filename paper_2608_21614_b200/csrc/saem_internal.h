@@ -13,7 +13,8 @@ namespace saem {
 constexpr int kTileRows = 128;              // weight rows per tile (the MMA M)
 constexpr int kTileK = 64;                  // reduction elements per tile (128 bytes of bf16)
 constexpr int kTileBytes = kTileRows * kTileK * 2;   // 16 KB
-constexpr int kMaxCtas = 160;               // upper bound of the persistent grid (B200: 148 SMs)
+constexpr int kMaxCtas = 320;               // upper bound of the persistent grid (two CTAs per SM on 148 SMs)
+constexpr int kMaxSms = 160;
 constexpr int kMaxNTile = 256;              // widest token tile (the MMA N)
 
 // Slot index per expert for one FFN launch; travels as a kernel parameter so that the residency
@@ -27,7 +28,7 @@ struct WorkspaceLayout {
     size_t status;        // int32 status word (+ padding)
     size_t counters;      // int32[2 * kMaxCtas] split-K arrival counters (gate/up, down)
     size_t h;             // bf16 [max_rows, d_ff]
-    size_t partials;      // fp32 [kMaxCtas][2][2][n_tile_max][128]
+    size_t partials;      // fp32 [CTAs][2][2][n_tile][128]: 2 CTAs/SM for n_tile <= 64, else 1 CTA/SM
     size_t logits, x, topk_idx, topk_w, counts, offsets, perm, inv_perm, x_packed, y_packed, shared_y, out;
     size_t total;
     int n_tile_max;
@@ -37,6 +38,29 @@ struct WorkspaceLayout {
 WorkspaceLayout workspace_layout(const saem_config& c);
 int validate_config(const saem_config* c);
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+
+// Launch with programmatic stream serialization: the kernel may start while the previous kernel of
+// the stream is still draining; every kernel launched this way executes `griddepcontrol.wait`
+// (pdl_wait) before it reads or writes anything a predecessor may touch.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
 
 // ---- kernel launchers (each returns a cudaError_t from the launch) ----
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
