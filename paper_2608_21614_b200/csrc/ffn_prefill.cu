@@ -1,0 +1,330 @@
+// Grouped SwiGLU expert FFN for LARGE segments (prefill, big decode batches): a real dense
+// contraction, so it is tiled for the tensor cores rather than for bytes (Sec. IV-E: one dense
+// batched execution per expert over its contiguous rows).
+//
+//   * Item: kPfTokens (128) tokens of one expert's segment (the MMA's M operand, loaded by TMA
+//     from x_packed / h; the code also supports two M tiles per item sharing each weight stage)
+//     x 256 weight rows (the N operand: for gate/up the 128 gate rows and the 128 up
+//     rows of one f-block, which the packed slot layout stores back to back; for the down
+//     projection two adjacent 128-row d-blocks) x 64 reduction elements per pipeline stage.
+//     tcgen05.mma 128x256x16, fp32 accumulators in TMEM: 256 columns per 128-token tile, a ring
+//     of two (512 columns) handed over tile by tile, so the epilogue of one tile overlaps the
+//     MMAs into the other.
+//   * gate and up land in the same accumulator tile (columns 0..127 and 128..255 of the same
+//     token lane), so SiLU(gate)*up is a per-thread operation and h is written once, bf16, with
+//     16-byte stores; y is written fp32 with 16-byte stores.
+//   * One persistent CTA per SM; whole tiles are dealt round-robin in the order (expert, weight
+//     block, token tile), so the CTAs that run at the same time share a weight block and it is
+//     fetched from HBM once and re-read from L2.  No tile is split, nothing is reduced across CTAs.
+//   * Warp roles and bounded mbarrier waits as in the streaming kernel (ffn_tensor.cu).
+#include "tc_common.cuh"
+
+namespace saem {
+
+constexpr int kPfThreads = 320;            // warp 0 copies, warp 1 MMA, warps 2..9 epilogue
+// Tokens per item.  128 = one MMA tile per item and four pipeline stages; 256 = two MMA tiles that
+// share every weight stage (a third fewer bytes per flop from L2, three stages, half as many
+// items).  Measured on the fine-grained 2048-token layer, 128 is faster: with a few hundred items
+// per launch the coarser items lose more to the last, partly filled round than they gain.
+constexpr int kPfTokens = 128;
+constexpr int kPfStageW = 2 * kTileBytes;  // 256 weight rows x 64 k
+constexpr int kPfStageX = kPfTokens * 128; // 256 tokens x 64 k
+constexpr int kPfStage = kPfStageW + kPfStageX;
+constexpr int kPfStages = kPfTokens == 128 ? 4 : 3;
+constexpr int kPfSmem = kPfStages * kPfStage + 1024;
+
+struct PfPlan {
+    int n_active;
+    int total_items;
+    int slot[SAEM_MAX_EXPERTS];
+    int row0[SAEM_MAX_EXPERTS];
+    int rows[SAEM_MAX_EXPERTS];
+    int item_base[SAEM_MAX_EXPERTS + 1];
+};
+
+struct PfItem {
+    int a, wb, mb;
+    int row_start, rows_here, n_cols;
+    int n_mt;               // 128-token MMA tiles in this item (1 or 2)
+};
+
+// item -> (active expert, weight block, token tile); weight block slowest, token tile fastest
+__device__ __forceinline__ void pf_decode(const PfPlan& plan, int it, int& cursor, int WB, int last_cols, PfItem& o) {
+    while (cursor + 1 < plan.n_active && plan.item_base[cursor + 1] <= it) ++cursor;
+    o.a = cursor;
+    const int local = it - plan.item_base[cursor];
+    const int m_blocks = (plan.rows[cursor] + kPfTokens - 1) / kPfTokens;
+    o.wb = local / m_blocks;
+    o.mb = local - o.wb * m_blocks;
+    o.row_start = plan.row0[cursor] + o.mb * kPfTokens;
+    const int left = plan.rows[cursor] - o.mb * kPfTokens;
+    o.rows_here = left < kPfTokens ? left : kPfTokens;
+    o.n_cols = (o.wb == WB - 1) ? last_cols : 256;
+    o.n_mt = o.rows_here > 128 ? 2 : 1;
+}
+
+// PHASE 0: h = silu(x Wg^T) * (x Wu^T);  PHASE 1: y = h Wd^T
+template <int PHASE>
+__global__ void __launch_bounds__(kPfThreads, 1)
+ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_constant__ CUtensorMap act_map) {
+    extern __shared__ uint8_t dyn_smem[];
+    __shared__ PfPlan plan;
+    __shared__ __align__(8) uint64_t bar_full[kPfStages], bar_empty[kPfStages], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_flag;
+    __shared__ int s_warp_act[kPfThreads / 32], s_warp_items[kPfThreads / 32];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int K = PHASE == 0 ? a.d : a.f;
+    const int KC = K / kTileK;
+    // weight blocks of 256 rows: gate/up -> one f-block (128 gate + 128 up rows); down -> two d-blocks
+    const int WB = PHASE == 0 ? a.f / kTileRows : (a.d / kTileRows + 1) / 2;
+    const int last_cols = PHASE == 0 ? 256 : ((a.d / kTileRows) & 1 ? 128 : 256);
+    const uint32_t smem_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < kPfStages; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_acc_full[s]), 1); mbar_init(smem_u32(&bar_acc_empty[s]), 8); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    pdl_wait();
+    pdl_launch_dependents();
+
+    // ---- plan (one thread per expert, block-wide prefix sums) ----
+    {
+        const int e = tid;
+        int rows = 0, r0 = 0;
+        if (e < a.E) {
+            int r1 = a.max_rows;
+            if (a.offsets) { r0 = a.offsets[e]; r1 = a.offsets[e + 1]; }
+            if (r1 > a.max_rows) r1 = a.max_rows;
+            rows = r1 > r0 ? r1 - r0 : 0;
+            if (!tab.in_subset[e]) rows = 0;
+            if (rows > 0 && tab.slot[e] < 0) {
+                if (blockIdx.x == 0) atomicExch(a.status, SAEM_ERR_NOT_RESIDENT);
+                rows = 0;
+            }
+        }
+        const int my_items = rows > 0 ? ((rows + kPfTokens - 1) / kPfTokens) * WB : 0;
+        int act_inc = rows > 0 ? 1 : 0, item_inc = my_items;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int na = __shfl_up_sync(0xffffffffu, act_inc, o), ni = __shfl_up_sync(0xffffffffu, item_inc, o);
+            if (lane >= o) { act_inc += na; item_inc += ni; }
+        }
+        if (lane == 31) { s_warp_act[warp] = act_inc; s_warp_items[warp] = item_inc; }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        int base_act = 0, base_items = 0, tot_act = 0, tot_items = 0;
+#pragma unroll
+        for (int w = 0; w < kPfThreads / 32; ++w) {
+            if (w < warp) { base_act += s_warp_act[w]; base_items += s_warp_items[w]; }
+            tot_act += s_warp_act[w];
+            tot_items += s_warp_items[w];
+        }
+        if (rows > 0) {
+            const int n = base_act + act_inc - 1;
+            plan.slot[n] = tab.slot[e];
+            plan.row0[n] = r0;
+            plan.rows[n] = rows;
+            plan.item_base[n] = base_items + item_inc - my_items;
+        }
+        if (tid == 0) {
+            plan.item_base[tot_act] = tot_items;
+            plan.n_active = tot_act;
+            plan.total_items = tot_items;
+        }
+        __syncthreads();
+    }
+    const uint32_t tmem_base = tmem_base_s;
+    const int total_items = plan.total_items;
+    const int G = gridDim.x;
+    volatile int* abort_p = &abort_flag;
+
+    if (warp == 0) {
+        // =============================== producer ===============================
+        int stage = 0, cursor = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        int issued = 0;
+        PfItem it;
+        for (int item = blockIdx.x; ok && item < total_items; item += G) {
+            pf_decode(plan, item, cursor, WB, last_cols, it);
+            const uint8_t* slot = a.slot_region + (size_t)plan.slot[it.a] * a.slot_bytes;
+            // gate/up: chunk (f-block, kc) is 32 KB (gate tile, up tile); down: tiles (2 wb, kc), (2 wb + 1, kc)
+            const uint8_t* w0 = PHASE == 0 ? slot + (size_t)it.wb * KC * kPfStageW
+                                           : slot + (size_t)2 * a.d * a.f * 2 + (size_t)(2 * it.wb) * KC * kTileBytes;
+            const uint8_t* w1 = PHASE == 0 ? w0 + kTileBytes : w0 + (size_t)KC * kTileBytes;
+            const size_t w_step = PHASE == 0 ? kPfStageW : kTileBytes;
+            const int n_boxes = (it.rows_here + 31) / 32;
+            const uint32_t w_bytes = it.n_cols == 256 ? kPfStageW : kTileBytes;
+            for (int kc = 0; kc < KC; ++kc) {
+                ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, a.status);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t full = smem_u32(&bar_full[stage]);
+                    const uint32_t ws = smem_base + (uint32_t)stage * kPfStage;
+                    mbar_expect_tx(full, w_bytes + (uint32_t)n_boxes * 4096u);
+                    bulk_g2s(ws, w0 + (size_t)kc * w_step, kTileBytes, full);
+                    if (it.n_cols == 256) bulk_g2s(ws + kTileBytes, w1 + (size_t)kc * w_step, kTileBytes, full);
+                    for (int b = 0; b < n_boxes; ++b)
+                        tma_2d(ws + kPfStageW + (uint32_t)b * 4096u, &act_map, kc * kTileK, it.row_start + b * 32, full);
+                }
+                ++issued;
+                if (++stage == kPfStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok && issued > 0) {     // let copies already in flight land before the CTA's memory goes away
+            unsigned long long t0 = globaltimer_ns();
+            while (globaltimer_ns() - t0 < 200000ull) {}
+        }
+    } else if (warp == 1) {
+        // =============================== MMA issuer ===============================
+        int stage = 0, acc = 0, cursor = 0;
+        uint32_t phase = 0, acc_phase[2] = {0u, 0u};
+        bool ok = true;
+        PfItem it;
+        for (int item = blockIdx.x; ok && item < total_items; item += G) {
+            pf_decode(plan, item, cursor, WB, last_cols, it);
+            const int acc0 = acc, acc1 = acc ^ 1;             // accumulators of the item's first / second tile
+            const uint32_t idesc = idesc_bf16(it.n_cols);
+            for (int kc = 0; ok && kc < KC; ++kc) {
+                ok = mbar_wait(smem_u32(&bar_full[stage]), phase, abort_p, a.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t ws = smem_base + (uint32_t)stage * kPfStage;
+                const uint32_t xs = ws + kPfStageW;
+                for (int t = 0; t < it.n_mt; ++t) {
+                    const int ac = t == 0 ? acc0 : acc1;
+                    if (kc == 0) {      // the accumulator must have been drained by the epilogue
+                        ok = mbar_wait(smem_u32(&bar_acc_empty[ac]), acc_phase[ac] ^ 1u, abort_p, a.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
+                    if (lane == 0) {
+                        const uint32_t d_tmem = tmem_base + (uint32_t)(ac * 256);
+#pragma unroll
+                        for (int k4 = 0; k4 < kTileK / 16; ++k4)
+                            tc_mma_bf16(d_tmem, smem_desc_sw128(xs + t * (kPfStageX / 2) + k4 * 32),
+                                        smem_desc_sw128(ws + k4 * 32), idesc, (kc > 0 || k4 > 0) ? 1u : 0u);
+                    }
+                }
+                if (!ok) break;
+                if (lane == 0) tc_commit(smem_u32(&bar_empty[stage]));
+                __syncwarp();
+                if (++stage == kPfStages) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            if (lane == 0) {
+                tc_commit(smem_u32(&bar_acc_full[acc0]));
+                if (it.n_mt == 2) tc_commit(smem_u32(&bar_acc_full[acc1]));
+            }
+            __syncwarp();
+            acc_phase[acc0] ^= 1u;
+            if (it.n_mt == 2) acc_phase[acc1] ^= 1u;
+            else acc ^= 1;                                    // a one-tile item takes one accumulator of the ring
+        }
+    } else {
+        // =============================== epilogue (warps 2..9) ===============================
+        const int q = warp & 3;                 // TMEM lane quarter = token rows 32q .. 32q+31
+        const int half = (warp - 2) >> 2;       // which half of the tile's columns
+        const int i = q * 32 + lane;            // token row inside the tile
+        int acc = 0, cursor = 0;
+        uint32_t acc_phase[2] = {0u, 0u};
+        bool ok = true;
+        PfItem it;
+        for (int item = blockIdx.x; ok && item < total_items; item += G) {
+            pf_decode(plan, item, cursor, WB, last_cols, it);
+            for (int t = 0; ok && t < it.n_mt; ++t) {
+                const int ac = t == 0 ? acc : acc ^ 1;
+                ok = mbar_wait(smem_u32(&bar_acc_full[ac]), acc_phase[ac], abort_p, a.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ac * 256);
+                const int r = t * 128 + i;
+                const bool valid = r < it.rows_here;
+                const size_t row = (size_t)(it.row_start + r);
+                if (PHASE == 0) {
+                    // h columns [64 half, 64 half + 64) of this f-block: gate at TMEM column c, up at 128 + c
+                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.h) + row * a.f + (size_t)it.wb * kTileRows;
+                    for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 16) {
+                        float g[16], u[16];
+                        tc_ld16(t_row + (uint32_t)c0, g);
+                        tc_ld16(t_row + (uint32_t)(128 + c0), u);
+                        if (valid) {
+                            uint32_t pk[8];
+#pragma unroll
+                            for (int n = 0; n < 8; ++n) {
+                                const float h0 = __fdividef(g[2 * n], 1.f + __expf(-g[2 * n])) * u[2 * n];
+                                const float h1 = __fdividef(g[2 * n + 1], 1.f + __expf(-g[2 * n + 1])) * u[2 * n + 1];
+                                __nv_bfloat162 p2 = __floats2bfloat162_rn(h0, h1);
+                                pk[n] = *reinterpret_cast<uint32_t*>(&p2);
+                            }
+                            uint4* o = reinterpret_cast<uint4*>(dst + c0);
+                            o[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            o[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        }
+                    }
+                } else {
+                    float* dst = a.y_packed + row * a.d + (size_t)it.wb * 256;
+                    const int c_half = it.n_cols / 2;
+                    for (int c0 = half * c_half; c0 < half * c_half + c_half; c0 += 16) {
+                        float v[16];
+                        tc_ld16(t_row + (uint32_t)c0, v);
+                        if (valid) {
+                            float4* o = reinterpret_cast<float4*>(dst + c0);
+#pragma unroll
+                            for (int n = 0; n < 4; ++n) o[n] = make_float4(v[4 * n], v[4 * n + 1], v[4 * n + 2], v[4 * n + 3]);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[ac]));
+                acc_phase[ac] ^= 1u;
+            }
+            if (it.n_mt == 1) acc ^= 1;
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    }
+}
+
+// ------------------------------------------------------------------------------------------- host
+static bool g_pf_init = false;
+
+cudaError_t ffn_prefill_init() {
+    if (g_pf_init) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(ffn_prefill_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(ffn_prefill_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmem);
+    if (e != cudaSuccess) return e;
+    g_pf_init = true;
+    return cudaSuccess;
+}
+
+cudaError_t launch_ffn_prefill(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x, const CUtensorMap& map_h,
+                               cudaStream_t st, int* n_launch) {
+    cudaError_t e = ffn_prefill_init();
+    if (e != cudaSuccess) return e;
+    const dim3 grid((unsigned)a.n_sm), block(kPfThreads);
+    e = launch_pdl(ffn_prefill_kernel<0>, grid, block, (size_t)kPfSmem, st, a, tab, map_x);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(ffn_prefill_kernel<1>, grid, block, (size_t)kPfSmem, st, a, tab, map_h);
+    *n_launch = 2;
+    return e;
+}
+
+}  // namespace saem

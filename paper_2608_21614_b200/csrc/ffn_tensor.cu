@@ -14,15 +14,12 @@
 //     k-range is split across CTAs is finished by whichever contributor arrives last, which adds
 //     the partial tiles in ascending CTA order -- deterministic, and no CTA ever waits for another.
 //   * Warp roles: warp 0 issues the copies, warp 1 issues tcgen05.mma into TMEM accumulators
-//     (double-buffered when they fit), warps 2..5 read TMEM back (tcgen05.ld), apply SiLU*up or
+//     (double-buffered when they fit), warps 2..9 read TMEM back (tcgen05.ld), apply SiLU*up or
 //     store y.  Stages are handed over with mbarriers; every wait is bounded and, when it runs out,
 //     sets SAEM_ERR_TIMEOUT in the device status word and makes the CTA drain and return.
 //
 // Two launches per FFN: gate/up (+SiLU*mul -> h, bf16) and down (-> y_packed, fp32).
-#include <cuda.h>
-#include <cuda_bf16.h>
-
-#include "saem_internal.h"
+#include "tc_common.cuh"
 
 namespace saem {
 
@@ -31,94 +28,7 @@ constexpr int kEpiThreads = 256;
 constexpr int kGateUpMaxTile = 128;           // widest token tile of the gate/up phase (two accumulator sets fit TMEM)
 constexpr int kMaxStages = 8;
 constexpr int kDynSmemMax = 220 * 1024;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 constexpr long long kSplitBelowItemsPerCta = 6;   // split items across CTAs only below this many items per CTA
-
-// ------------------------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-// Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit runs out or
-// another role of this CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    unsigned long long t0 = 0;
-    for (uint32_t i = 0;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 1023u) == 1023u) {
-            if (*abort_flag) return false;
-            unsigned long long now = globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicExch(status, SAEM_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 bytes apart,
-// 8-row groups 1024 bytes apart (the layout both the packed weight tiles and the TMA boxes have).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t idesc_bf16(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
-}
 
 // --------------------------------------------------------------------------------------- the plan
 struct Plan {
@@ -140,29 +50,43 @@ struct Item {
 
 struct ItemWalker {
     const Plan* plan;
-    long long c, c1;        // next chunk, end of this CTA's range
+    long long c, c1;        // next chunk, end of this CTA's range (contiguous mode)
+    long long stride;       // > 0: whole items it, it + stride, ... < c1 (c, c1 then count items)
     int KC, RB, n_tile;
     int a_cursor;
-    __device__ __forceinline__ ItemWalker(const Plan* p, long long c0_, long long c1_, int KC_, int RB_, int nt)
-        : plan(p), c(c0_), c1(c1_), KC(KC_), RB(RB_), n_tile(nt), a_cursor(0) {}
+    __device__ __forceinline__ ItemWalker(const Plan* p, long long c0_, long long c1_, long long stride_, int KC_,
+                                          int RB_, int nt)
+        : plan(p), c(c0_), c1(c1_), stride(stride_), KC(KC_), RB(RB_), n_tile(nt), a_cursor(0) {}
     __device__ __forceinline__ bool next(Item& o) {
         if (c >= c1) return false;
-        long long it = c / KC;
+        long long it;
+        if (stride > 0) {
+            it = c;
+            o.kc_begin = 0;
+            o.kc_end = KC;
+            c += stride;
+        } else {
+            it = c / KC;
+            o.kc_begin = (int)(c - it * KC);
+            long long end = (it + 1) * KC;
+            if (end > c1) end = c1;
+            o.kc_end = (int)(end - it * KC);
+            c = end;
+        }
         o.it = it;
-        o.kc_begin = (int)(c - it * KC);
-        long long end = (it + 1) * KC;
-        if (end > c1) end = c1;
-        o.kc_end = (int)(end - it * KC);
         while (a_cursor + 1 < plan->n_active && plan->item_base[a_cursor + 1] <= it) ++a_cursor;
         o.a = a_cursor;
-        int local = (int)(it - plan->item_base[a_cursor]);
-        o.nb = local / RB;
-        o.rb = local - o.nb * RB;
+        // items of one expert: weight-row block slowest, token tile fastest, so that the token
+        // tiles that share a weight block are worked on at the same time by neighbouring CTAs
+        // (whole-item mode deals items round-robin) and the block is fetched from HBM once
+        const int local = (int)(it - plan->item_base[a_cursor]);
+        const int n_blocks = (plan->rows[a_cursor] + n_tile - 1) / n_tile;
+        o.rb = local / n_blocks;
+        o.nb = local - o.rb * n_blocks;
         o.row_start = plan->row0[a_cursor] + o.nb * n_tile;
         int left = plan->rows[a_cursor] - o.nb * n_tile;
         o.rows_here = left < n_tile ? left : n_tile;
         o.n_eff = (o.rows_here + 15) & ~15;
-        c = end;
         return true;
     }
 };
@@ -269,14 +193,14 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     const long long total_chunks = (long long)plan.total_items * KC;
     const long long G = gridDim.x;
     const bool split_k = (long long)plan.total_items < kSplitBelowItemsPerCta * G;
-    const long long c0 = split_k ? total_chunks * blockIdx.x / G : ((long long)plan.total_items * blockIdx.x / G) * KC;
-    const long long c1 = split_k ? total_chunks * (blockIdx.x + 1) / G
-                                 : ((long long)plan.total_items * (blockIdx.x + 1) / G) * KC;
+    const long long c0 = split_k ? total_chunks * blockIdx.x / G : (long long)blockIdx.x;
+    const long long c1 = split_k ? total_chunks * (blockIdx.x + 1) / G : (long long)plan.total_items;
+    const long long walk_stride = split_k ? 0 : G;
     volatile int* abort_p = &abort_flag;
 
     if (warp == 0) {
         // =============================== producer ===============================
-        ItemWalker walk(&plan, c0, c1, KC, RB, n_tile);
+        ItemWalker walk(&plan, c0, c1, walk_stride, KC, RB, n_tile);
         Item it;
         int stage = 0;
         uint32_t phase = 0;
@@ -310,7 +234,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
         }
     } else if (warp == 1) {
         // =============================== MMA issuer ===============================
-        ItemWalker walk(&plan, c0, c1, KC, RB, n_tile);
+        ItemWalker walk(&plan, c0, c1, walk_stride, KC, RB, n_tile);
         Item it;
         int stage = 0, acc = 0;
         uint32_t phase = 0, acc_phase[2] = {0u, 0u};
@@ -354,7 +278,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
         const int half = (warp - 2) >> 2;
         const int i = q * 32 + lane;            // weight row inside the tile
         const int epi_tid = tid - 64;
-        ItemWalker walk(&plan, c0, c1, KC, RB, n_tile);
+        ItemWalker walk(&plan, c0, c1, walk_stride, KC, RB, n_tile);
         Item it;
         int acc = 0;
         uint32_t acc_phase[2] = {0u, 0u};
@@ -523,6 +447,8 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
     alignas(64) CUtensorMap map_x, map_h;
     if (!make_act_map(&map_x, a.x_packed, a.max_rows, a.d, box_rows)) return cudaErrorInvalidValue;
     if (!make_act_map(&map_h, a.h, a.max_rows, a.f, box_rows)) return cudaErrorInvalidValue;
+    // Segments that can exceed 64 rows are a dense contraction: tile them for the tensor cores.
+    if (a.n_tile > 64) return launch_ffn_prefill(a, tab, map_x, map_h, st, n_launch);
     // Small token tiles (decode): two CTAs per SM, each with half the shared memory, so that one
     // CTA's prologue, epilogue and split-item reduction overlap the other's streaming.
     const bool two_per_sm = a.n_tile <= 64;
