@@ -26,6 +26,7 @@
  *     bounded wait that ran out) set a sticky device status word, read by
  *     saem_last_device_status(); kernels never trap and never wait without a bound.
  *   - The four step calls never synchronise and never read device results on the host.
+ *   - A context is not thread-safe: calls on one context must come from one thread at a time.
  */
 #ifndef SAEM_H_
 #define SAEM_H_
@@ -64,8 +65,16 @@ enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2 };
  * temporary slots shared by all layers (Sec. VI ablation: on-demand loads through a reserved
  * temporary slot).  renorm: 1 = softmax over the k selected logits (weights sum to 1), 0 = the
  * selected experts' probabilities under the softmax over all experts.  out_dtype: SAEM_OUT_*.
- * ffn_path: SAEM_FFN_AUTO picks the tensor-core streaming kernels; SAEM_FFN_SCALAR forces the
- * plain scalar kernels (kept for triage).
+ * ffn_path: SAEM_FFN_AUTO picks the tensor-core kernels; SAEM_FFN_SCALAR forces the plain scalar
+ * kernels (kept for triage).
+ * n_shared (0..16, n_experts + n_shared <= SAEM_MAX_EXPERTS): always-on shared experts of the same
+ * width d_ff that run INSIDE the layer's grouped launch.  They are experts n_experts ..
+ * n_experts + n_shared - 1 of every layer for the cache calls (outside the routed cache-ratio
+ * budget: give them slots); saem_repack appends one segment of all T tokens per shared expert
+ * after the T*top_k pair rows (counts, offsets get n_shared more entries; x_packed, y_packed
+ * hold T*(top_k + n_shared) rows); saem_combine adds their outputs with weight 1.  A shared
+ * expert of width m*d_ff is m such experts (the down projection sums over the hidden units).
+ * Shared experts of another width use a second context instead (see saem_moe_step).
  */
 typedef struct saem_config {
     int32_t d_model;
@@ -79,7 +88,7 @@ typedef struct saem_config {
     int32_t renorm;
     int32_t out_dtype;
     int32_t ffn_path;
-    int32_t reserved;
+    int32_t n_shared;
 } saem_config;
 
 /* Library version (major*10000 + minor*100 + patch) and a static string for a status code. */
@@ -144,7 +153,8 @@ int saem_repack(saem_ctx* ctx, const int32_t* topk_idx, const void* x, int T, in
  * accumulation, hidden activations rounded to bf16 in the context's workspace, y_packed[max_rows,
  * d_model] fp32 (dev).  Weights come from the slots that `layer`'s residency map (or a temporary
  * slot) gives.  offsets (dev) is read on the device only; max_rows bounds offsets[n_experts] and
- * must not exceed max_tokens * top_k.
+ * must not exceed max_tokens * top_k.  offsets may be NULL only when n_experts == 1: the single
+ * segment is then rows [0, max_rows) (used for always-on shared experts, whose input is x itself).
  *   expert_subset (host, may be NULL): run only these experts (rows of the others are left
  *   untouched).  With a subset, an expert that has no slot returns NOT_RESIDENT before any
  *   enqueue.  Without one, experts without a slot are skipped on the device; if such an expert has

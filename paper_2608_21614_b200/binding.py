@@ -27,7 +27,7 @@ SAEM_FFN_AUTO, SAEM_FFN_SCALAR, SAEM_FFN_TENSOR = 0, 1, 2
 class saem_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "d_model", "d_ff", "n_experts", "top_k", "max_tokens", "n_layers", "slots_per_layer", "temp_slots",
-        "renorm", "out_dtype", "ffn_path", "reserved")]
+        "renorm", "out_dtype", "ffn_path", "n_shared")]
 
 
 class SaemError(RuntimeError):
@@ -267,10 +267,10 @@ def saem_expert_ffn_static(x_packed, offsets, n_experts, max_rows, d_model, d_ff
 
 # ------------------------------------------------------------------------- memory plumbing (torch)
 def make_config(d_model, d_ff, n_experts, top_k, max_tokens, n_layers=1, slots_per_layer=None, temp_slots=0,
-                renorm=1, out_dtype=SAEM_OUT_F32, ffn_path=SAEM_FFN_AUTO) -> saem_config:
+                renorm=1, out_dtype=SAEM_OUT_F32, ffn_path=SAEM_FFN_AUTO, n_shared=0) -> saem_config:
     return saem_config(d_model, d_ff, n_experts, top_k, max_tokens, n_layers,
-                       n_experts if slots_per_layer is None else slots_per_layer, temp_slots, renorm, out_dtype,
-                       ffn_path, 0)
+                       n_experts + n_shared if slots_per_layer is None else slots_per_layer, temp_slots, renorm,
+                       out_dtype, ffn_path, n_shared)
 
 
 class Context:

@@ -11,7 +11,7 @@ namespace saem {
 
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ inv_perm, const float* __restrict__ w,
-               int T, int k, int d, const float* __restrict__ shared_y, void* __restrict__ out, int out_bf16) {
+               int T, int k, int S, int d, const float* __restrict__ shared_y, void* __restrict__ out, int out_bf16) {
     pdl_wait();
     pdl_launch_dependents();
     const int vec_per_row = d >> 2;
@@ -30,6 +30,10 @@ combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ inv_perm
             acc.z = fmaf(wj, v.z, acc.z);
             acc.w = fmaf(wj, v.w, acc.w);
         }
+        for (int sh = 0; sh < S; ++sh) {               // in-layer shared experts: rows after the T*k pairs
+            const float4 v = *reinterpret_cast<const float4*>(y + ((size_t)T * k + (size_t)sh * T + t) * d + (size_t)c4 * 4);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
         if (shared_y) {
             const float4 s = *reinterpret_cast<const float4*>(shared_y + (size_t)t * d + (size_t)c4 * 4);
             acc.x += s.x; acc.y += s.y; acc.z += s.z; acc.w += s.w;
@@ -46,12 +50,12 @@ combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ inv_perm
     }
 }
 
-cudaError_t launch_combine(const float* y, const int32_t* inv_perm, const float* w, int T, int k, int d,
+cudaError_t launch_combine(const float* y, const int32_t* inv_perm, const float* w, int T, int k, int S, int d,
                            const float* shared_y, void* out, int out_bf16, cudaStream_t st) {
     long long total = (long long)T * (d / 4);
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    return launch_pdl(combine_kernel, dim3((unsigned)blocks), dim3(256), 0, st, y, inv_perm, w, T, k, d, shared_y, out,
+    return launch_pdl(combine_kernel, dim3((unsigned)blocks), dim3(256), 0, st, y, inv_perm, w, T, k, S, d, shared_y, out,
                       out_bf16);
 }
 

@@ -25,7 +25,7 @@ struct RepackSmem {
 };
 
 // Shared-memory carve: [RepackSmem][chunk table uint16 n_chunks*E][rank uint8 P_padded][perm int32 P (fused only)]
-__device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int P, int E, RepackSmem& sm,
+__device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int P, int E, int S, int T, RepackSmem& sm,
                                             uint16_t* table, uint8_t* rank, int32_t* perm_s, bool write_global,
                                             int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                                             int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
@@ -77,6 +77,9 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
     if (write_global) {
         for (int e = tid; e < E; e += blockDim.x) counts[e] = sm.counts[e];
         for (int e = tid; e <= E; e += blockDim.x) offsets[e] = sm.offsets[e];
+        // in-layer shared experts: one segment of all T tokens each, after the T*k pair rows
+        if (S > 0 && tid == 0) offsets[E] = P;
+        for (int sh = tid; sh < S; sh += blockDim.x) { counts[E + sh] = T; offsets[E + sh + 1] = P + (sh + 1) * T; }
         if (tid == 0 && sm.bad) atomicExch(status, SAEM_ERR_INVALID_ARG);
     }
     for (int p = tid; p < P; p += blockDim.x) {
@@ -97,7 +100,7 @@ __device__ __forceinline__ void copy_row(const uint16_t* __restrict__ src, uint1
 }
 
 __global__ void __launch_bounds__(kRepackThreads)
-repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict__ x, int T, int E, int k, int d,
+repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict__ x, int T, int E, int S, int k, int d,
                     int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ perm,
                     int32_t* __restrict__ inv_perm, uint16_t* __restrict__ x_packed, int* __restrict__ status) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -110,7 +113,7 @@ repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict_
     int32_t* perm_s = reinterpret_cast<int32_t*>(smem_raw + off);
     uint8_t* rank = smem_raw + off + (size_t)n_chunks * 32 * 4;
     for (int i = threadIdx.x; i < n_chunks * 32; i += blockDim.x) perm_s[i] = -1;
-    index_phase(idx, P, E, sm, table, rank, perm_s, blockIdx.x == 0, counts, offsets, perm, inv_perm, status);
+    index_phase(idx, P, E, S, T, sm, table, rank, perm_s, blockIdx.x == 0, counts, offsets, perm, inv_perm, status);
     const int total = sm.offsets[E];                 // rows actually packed (pairs with a valid expert)
     // each CTA copies rows r = blockIdx.x, blockIdx.x + gridDim.x, ...; 128 threads per row
     const int sub = threadIdx.x >> 7, nsub = blockDim.x >> 7;
@@ -118,10 +121,12 @@ repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict_
         int p = perm_s[r];
         copy_row(x + (size_t)(p / k) * d, x_packed + (size_t)r * d, d, threadIdx.x & 127, 128);
     }
+    for (int r = blockIdx.x * nsub + sub; r < S * T; r += gridDim.x * nsub)      // shared segments: x itself
+        copy_row(x + (size_t)(r % T) * d, x_packed + (size_t)(P + r) * d, d, threadIdx.x & 127, 128);
 }
 
 __global__ void __launch_bounds__(1024)
-repack_index_kernel(const int32_t* __restrict__ idx, int T, int E, int k, int32_t* __restrict__ counts,
+repack_index_kernel(const int32_t* __restrict__ idx, int T, int E, int S, int k, int32_t* __restrict__ counts,
                     int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
                     int* __restrict__ status) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -131,23 +136,26 @@ repack_index_kernel(const int32_t* __restrict__ idx, int T, int E, int k, int32_
     RepackSmem& sm = *reinterpret_cast<RepackSmem*>(smem_raw);
     uint16_t* table = reinterpret_cast<uint16_t*>(smem_raw + sizeof(RepackSmem));
     uint8_t* rank = smem_raw + sizeof(RepackSmem) + (((size_t)n_chunks * E * 2 + 15) & ~(size_t)15);
-    index_phase(idx, P, E, sm, table, rank, nullptr, true, counts, offsets, perm, inv_perm, status);
+    index_phase(idx, P, E, S, T, sm, table, rank, nullptr, true, counts, offsets, perm, inv_perm, status);
 }
 
 __global__ void __launch_bounds__(256)
 repack_gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__ perm,
-                     const int32_t* __restrict__ offsets, int E, int k, int d, uint16_t* __restrict__ x_packed) {
+                     const int32_t* __restrict__ offsets, int T, int E, int S, int k, int d,
+                     uint16_t* __restrict__ x_packed) {
     pdl_wait();
     pdl_launch_dependents();
-    const int total = offsets[E];
+    const int total = S > 0 ? T * k : offsets[E];
     const int sub = threadIdx.x >> 6, nsub = blockDim.x >> 6;     // 64 threads per row
     for (int r = blockIdx.x * nsub + sub; r < total; r += gridDim.x * nsub) {
         int p = perm[r];
         copy_row(x + (size_t)(p / k) * d, x_packed + (size_t)r * d, d, threadIdx.x & 63, 64);
     }
+    for (int r = blockIdx.x * nsub + sub; r < S * T; r += gridDim.x * nsub)      // shared segments: x itself
+        copy_row(x + (size_t)(r % T) * d, x_packed + (size_t)(T * k + r) * d, d, threadIdx.x & 63, 64);
 }
 
-cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, int k, int d, int32_t* counts,
+cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, int S, int k, int d, int32_t* counts,
                           int32_t* offsets, int32_t* perm, int32_t* inv_perm, uint16_t* x_packed, int* status,
                           int n_sm, cudaStream_t st, int* n_launch) {
     const int P = T * k, n_chunks = (P + 31) >> 5;
@@ -163,19 +171,19 @@ cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, i
     if (P <= kFusedPairs) {
         size_t smem = base + (size_t)n_chunks * 32 * 4 + (size_t)n_chunks * 32;
         int rows_per_cta = kRepackThreads / 128;
-        int grid = (P + rows_per_cta - 1) / rows_per_cta;
+        int grid = (P + S * T + rows_per_cta - 1) / rows_per_cta;
         if (grid < 1) grid = 1;
         if (grid > n_sm) grid = n_sm;
         *n_launch = 1;
-        return launch_pdl(repack_fused_kernel, dim3(grid), dim3(kRepackThreads), smem, st, idx, x, T, E, k, d, counts,
-                          offsets, perm, inv_perm, x_packed, status);
+        return launch_pdl(repack_fused_kernel, dim3(grid), dim3(kRepackThreads), smem, st, idx, x, T, E, S, k, d,
+                          counts, offsets, perm, inv_perm, x_packed, status);
     }
     size_t smem = base + (size_t)n_chunks * 32;
-    cudaError_t e = launch_pdl(repack_index_kernel, dim3(1), dim3(1024), smem, st, idx, T, E, k, counts, offsets, perm,
+    cudaError_t e = launch_pdl(repack_index_kernel, dim3(1), dim3(1024), smem, st, idx, T, E, S, k, counts, offsets, perm,
                                inv_perm, status);
     if (e != cudaSuccess) return e;
     *n_launch = 2;
-    return launch_pdl(repack_gather_kernel, dim3(n_sm * 4), dim3(256), 0, st, x, perm, offsets, E, k, d, x_packed);
+    return launch_pdl(repack_gather_kernel, dim3(n_sm * 4), dim3(256), 0, st, x, perm, offsets, T, E, S, k, d, x_packed);
 }
 
 }  // namespace saem

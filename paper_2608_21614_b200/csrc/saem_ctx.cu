@@ -18,7 +18,8 @@ int validate_config(const saem_config* c) {
     if (c->n_experts < 1 || c->n_experts > SAEM_MAX_EXPERTS) return SAEM_ERR_SHAPE;
     if (c->top_k < 1 || c->top_k > c->n_experts) return SAEM_ERR_SHAPE;
     if (c->max_tokens < 1 || (long long)c->max_tokens * c->top_k > 65535) return SAEM_ERR_SHAPE;
-    if (c->n_layers < 1 || c->slots_per_layer < 0 || c->slots_per_layer > c->n_experts) return SAEM_ERR_SHAPE;
+    if (c->n_shared < 0 || c->n_shared > 16 || c->n_experts + c->n_shared > SAEM_MAX_EXPERTS) return SAEM_ERR_SHAPE;
+    if (c->n_layers < 1 || c->slots_per_layer < 0 || c->slots_per_layer > c->n_experts + c->n_shared) return SAEM_ERR_SHAPE;
     if (c->temp_slots < 0 || c->temp_slots > 4096) return SAEM_ERR_SHAPE;
     if ((long long)c->n_layers * c->slots_per_layer + c->temp_slots < 1) return SAEM_ERR_SHAPE;
     if (c->out_dtype != SAEM_OUT_F32 && c->out_dtype != SAEM_OUT_BF16) return SAEM_ERR_INVALID_ARG;
@@ -32,7 +33,9 @@ int validate_config(const saem_config* c) {
 WorkspaceLayout workspace_layout(const saem_config& c) {
     WorkspaceLayout L{};
     const size_t A = 1024;
-    size_t P = (size_t)c.max_tokens * c.top_k, T = c.max_tokens, d = c.d_model, f = c.d_ff, E = c.n_experts;
+    size_t P = (size_t)c.max_tokens * c.top_k, T = c.max_tokens, d = c.d_model, f = c.d_ff;
+    size_t E = (size_t)c.n_experts + c.n_shared;            // experts with a segment: routed, then shared
+    size_t R = P + (size_t)c.n_shared * T;                  // packed rows: pairs, then T rows per shared expert
     int nt = round_up(c.max_tokens < kMaxNTile ? c.max_tokens : kMaxNTile, 16);
     L.n_tile_max = nt;
     L.partial_slot_floats = (size_t)2 * nt * kTileRows;
@@ -40,13 +43,13 @@ WorkspaceLayout workspace_layout(const saem_config& c) {
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, A); return o; };
     L.status = take(256);
     L.counters = take(sizeof(int) * 2 * kMaxCtas);
-    L.h = take(P * f * 2);
+    L.h = take(R * f * 2);
     {   // split-K partial tiles: the larger of the two launch shapes (see launch_ffn_tensor)
         size_t small_tile = (size_t)2 * (nt < 64 ? nt : 64) * kTileRows;
         size_t a = (size_t)kMaxCtas * 2 * small_tile, b = (size_t)kMaxSms * 2 * L.partial_slot_floats;
         L.partials = take((a > b ? a : b) * sizeof(float));
     }
-    L.logits = take(T * E * 4);
+    L.logits = take(T * (size_t)c.n_experts * 4);
     L.x = take(T * d * 2);
     L.topk_idx = take(P * 4);
     L.topk_w = take(P * 4);
@@ -54,8 +57,8 @@ WorkspaceLayout workspace_layout(const saem_config& c) {
     L.offsets = take((E + 1) * 4);
     L.perm = take(P * 4);
     L.inv_perm = take(P * 4);
-    L.x_packed = take(P * d * 2);
-    L.y_packed = take(P * d * 4);
+    L.x_packed = take(R * d * 2);
+    L.y_packed = take(R * d * 4);
     L.shared_y = take(T * d * 4);
     L.out = take(T * d * 4);
     L.total = off;
@@ -140,9 +143,10 @@ int saem_create(const saem_config* cfg, void* slot_region, size_t slot_region_by
     c->n_fixed_slots = cfg->n_layers * cfg->slots_per_layer;
     c->next_temp = 0;
     c->launches = 0;
-    c->dynamic_residency = cfg->slots_per_layer < cfg->n_experts || cfg->temp_slots > 0;
+    c->n_total = cfg->n_experts + cfg->n_shared;
+    c->dynamic_residency = cfg->slots_per_layer < c->n_total || cfg->temp_slots > 0;
     int n_slots = c->n_fixed_slots + cfg->temp_slots;
-    size_t LE = (size_t)cfg->n_layers * cfg->n_experts;
+    size_t LE = (size_t)cfg->n_layers * c->n_total;
     c->slot_of = (int32_t*)malloc(sizeof(int32_t) * LE);
     c->temp_of = (int32_t*)malloc(sizeof(int32_t) * LE);
     c->slot_owner = (int32_t*)malloc(sizeof(int32_t) * n_slots);
@@ -152,6 +156,8 @@ int saem_create(const saem_config* cfg, void* slot_region, size_t slot_region_by
     c->read_ev = (cudaEvent_t*)calloc(cfg->n_layers, sizeof(cudaEvent_t));
     c->read_recorded = (uint8_t*)calloc(cfg->n_layers, 1);
     c->temp_last_layer = (int32_t*)malloc(sizeof(int32_t) * (cfg->temp_slots > 0 ? cfg->temp_slots : 1));
+    c->last_stream = (cudaStream_t*)calloc(cfg->n_layers, sizeof(cudaStream_t));
+    c->ffn_seen = (uint8_t*)calloc(cfg->n_layers, 1);
     c->pinned_status = nullptr;
     for (size_t i = 0; i < LE; ++i) c->slot_of[i] = c->temp_of[i] = -1;
     for (int i = 0; i < n_slots; ++i) c->slot_owner[i] = -1;
@@ -188,7 +194,7 @@ void saem_destroy(saem_ctx* c) {
             if (c->read_ev[i]) cudaEventDestroy(c->read_ev[i]);
     if (c->pinned_status) cudaFreeHost(c->pinned_status);
     free(c->slot_of); free(c->temp_of); free(c->slot_owner); free(c->ready_ev); free(c->ev_pending);
-    free(c->ev_recorded); free(c->read_ev); free(c->read_recorded); free(c->temp_last_layer);
+    free(c->ev_recorded); free(c->read_ev); free(c->read_recorded); free(c->temp_last_layer); free(c->last_stream); free(c->ffn_seen);
     delete c;
 }
 
@@ -249,7 +255,7 @@ int saem_repack(saem_ctx* c, const int32_t* idx, const void* x, int T, int32_t* 
     if (T > 0 && (!idx || !x || !perm || !inv_perm || !x_packed)) return SAEM_ERR_INVALID_ARG;
     if (misaligned(x) || misaligned(x_packed)) return SAEM_ERR_ALIGNMENT;
     int nl = 0;
-    CUDA_TRY(launch_repack(idx, (const uint16_t*)x, T, c->cfg.n_experts, c->cfg.top_k, c->cfg.d_model, counts,
+    CUDA_TRY(launch_repack(idx, (const uint16_t*)x, T, c->cfg.n_experts, c->cfg.n_shared, c->cfg.top_k, c->cfg.d_model, counts,
                            offsets, perm, inv_perm, (uint16_t*)x_packed, (int*)(c->ws + c->lay.status), c->n_sm,
                            (cudaStream_t)stream, &nl));
     c->launches += nl;
@@ -261,31 +267,32 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     if (!c) return SAEM_ERR_INVALID_ARG;
     const saem_config& g = c->cfg;
     if (layer < 0 || layer >= g.n_layers) return SAEM_ERR_INVALID_ARG;
-    if (max_rows < 0 || max_rows > g.max_tokens * g.top_k) return SAEM_ERR_SHAPE;
+    if (max_rows < 0 || max_rows > g.max_tokens * (g.top_k + g.n_shared)) return SAEM_ERR_SHAPE;
     if (max_rows == 0) return SAEM_OK;
     if (!x_packed || !y_packed) return SAEM_ERR_INVALID_ARG;
-    if (!offsets && g.n_experts != 1) return SAEM_ERR_INVALID_ARG;
+    const int ES = c->n_total;
+    if (!offsets && ES != 1) return SAEM_ERR_INVALID_ARG;
     if (misaligned(x_packed) || misaligned(y_packed)) return SAEM_ERR_ALIGNMENT;
     if (subset && n_subset < 0) return SAEM_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
 
     SlotTable tab;
-    const int32_t* so = c->slot_of + (size_t)layer * g.n_experts;
-    const int32_t* to = c->temp_of + (size_t)layer * g.n_experts;
+    const int32_t* so = c->slot_of + (size_t)layer * ES;
+    const int32_t* to = c->temp_of + (size_t)layer * ES;
     for (int e = 0; e < SAEM_MAX_EXPERTS; ++e) { tab.slot[e] = -1; tab.in_subset[e] = 0; }
     auto resolve = [&](int e) { return so[e] >= 0 ? so[e] : to[e]; };
     if (subset) {
         for (int i = 0; i < n_subset; ++i) {
             int e = subset[i];
-            if (e < 0 || e >= g.n_experts) return SAEM_ERR_INVALID_ARG;
+            if (e < 0 || e >= ES) return SAEM_ERR_INVALID_ARG;
             if (resolve(e) < 0) return SAEM_ERR_NOT_RESIDENT;
         }
         for (int i = 0; i < n_subset; ++i) { tab.slot[subset[i]] = resolve(subset[i]); tab.in_subset[subset[i]] = 1; }
     } else {
-        for (int e = 0; e < g.n_experts; ++e) { tab.slot[e] = resolve(e); tab.in_subset[e] = 1; }
+        for (int e = 0; e < ES; ++e) { tab.slot[e] = resolve(e); tab.in_subset[e] = 1; }
     }
     // order this stream after loads still in flight for the slots it may read
-    for (int e = 0; e < g.n_experts; ++e) {
+    for (int e = 0; e < ES; ++e) {
         int s = tab.slot[e];
         if (s < 0 || !c->ev_pending[s]) continue;
         cudaError_t q = cudaEventQuery(c->ready_ev[s]);
@@ -298,7 +305,7 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     a.x_packed = (const uint16_t*)x_packed;
     a.offsets = offsets;
     a.max_rows = max_rows;
-    a.E = g.n_experts; a.d = g.d_model; a.f = g.d_ff;
+    a.E = ES; a.d = g.d_model; a.f = g.d_ff;
     a.slot_region = c->slot_region;
     a.slot_bytes = c->slot_bytes;
     a.h = (uint16_t*)(c->ws + c->lay.h);
@@ -316,10 +323,12 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
         CUDA_TRY(launch_ffn_tensor(a, tab, st, &nl));
     }
     c->launches += nl;
+    c->last_stream[layer] = st;
+    c->ffn_seen[layer] = 1;
     if (c->dynamic_residency) {
         CUDA_TRY(cudaEventRecord(c->read_ev[layer], st));
         c->read_recorded[layer] = 1;
-        for (int e = 0; e < g.n_experts; ++e) {
+        for (int e = 0; e < ES; ++e) {
             int s = tab.slot[e];
             if (s >= c->n_fixed_slots) c->temp_last_layer[s - c->n_fixed_slots] = layer;
         }
@@ -334,7 +343,7 @@ int saem_combine(saem_ctx* c, const float* y, const int32_t* inv_perm, const flo
     if (T == 0) return SAEM_OK;
     if (!y || !inv_perm || !w || !out) return SAEM_ERR_INVALID_ARG;
     if (misaligned(y) || misaligned(out) || misaligned(shared_y)) return SAEM_ERR_ALIGNMENT;
-    CUDA_TRY(launch_combine(y, inv_perm, w, T, c->cfg.top_k, c->cfg.d_model, shared_y, out,
+    CUDA_TRY(launch_combine(y, inv_perm, w, T, c->cfg.top_k, c->cfg.n_shared, c->cfg.d_model, shared_y, out,
                             c->cfg.out_dtype == SAEM_OUT_BF16, (cudaStream_t)stream));
     c->launches += 1;
     return SAEM_OK;
@@ -370,7 +379,7 @@ int saem_moe_step(saem_ctx* c, saem_ctx* sh, int layer, const float* logits, con
     if ((s = saem_route(c, logits, T, idx, tw, stream)) != SAEM_OK) return s;
     if ((s = saem_repack(c, idx, x, T, (int32_t*)(w + L.counts), offsets, (int32_t*)(w + L.perm), inv,
                          w + L.x_packed, stream)) != SAEM_OK) return s;
-    if ((s = saem_expert_ffn(c, layer, w + L.x_packed, offsets, T * g.top_k, nullptr, 0, y, stream)) != SAEM_OK)
+    if ((s = saem_expert_ffn(c, layer, w + L.x_packed, offsets, T * (g.top_k + g.n_shared), nullptr, 0, y, stream)) != SAEM_OK)
         return s;
     if (sh && (s = saem_expert_ffn(sh, layer, x, nullptr, T, nullptr, 0, shy, stream)) != SAEM_OK) return s;
     return saem_combine(c, y, inv, tw, T, sh ? shy : nullptr, out, stream);
@@ -399,7 +408,7 @@ int saem_moe_step_host(saem_ctx* c, saem_ctx* sh, int layer, const float* logits
 // ------------------------------------------------------------------------------------------- cache
 static int check_le(saem_ctx* c, int layer, int expert) {
     if (!c) return SAEM_ERR_INVALID_ARG;
-    if (layer < 0 || layer >= c->cfg.n_layers || expert < 0 || expert >= c->cfg.n_experts) return SAEM_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= c->cfg.n_layers || expert < 0 || expert >= c->n_total) return SAEM_ERR_INVALID_ARG;
     return SAEM_OK;
 }
 
@@ -408,7 +417,7 @@ int saem_cache_load(saem_ctx* c, int layer, int expert, int slot, const void* pi
     if (s != SAEM_OK) return s;
     if (!pinned) return SAEM_ERR_INVALID_ARG;
     const saem_config& g = c->cfg;
-    size_t le = (size_t)layer * g.n_experts + expert;
+    size_t le = (size_t)layer * c->n_total + expert;
     cudaStream_t cs = (cudaStream_t)copy_stream;
     int gslot;
     int wait_layer = -1;
@@ -432,7 +441,12 @@ int saem_cache_load(saem_ctx* c, int layer, int expert, int slot, const void* pi
     }
     c->slot_owner[gslot] = (int32_t)le;
     // the copy must not overtake an enqueued FFN that still reads the slot's previous content
-    if (wait_layer >= 0 && c->read_recorded[wait_layer]) {
+    if (wait_layer >= 0 && !c->read_recorded[wait_layer] && c->ffn_seen[wait_layer]) {
+        // fully resident configurations record no event per FFN: mark the tail of that layer's
+        // compute stream now (everything enqueued so far, hence every FFN that reads the slot)
+        if (cudaEventRecord(c->read_ev[wait_layer], c->last_stream[wait_layer]) != cudaSuccess) return SAEM_ERR_CUDA;
+        if (cudaStreamWaitEvent(cs, c->read_ev[wait_layer], 0) != cudaSuccess) return SAEM_ERR_CUDA;
+    } else if (wait_layer >= 0 && c->read_recorded[wait_layer]) {
         if (cudaStreamWaitEvent(cs, c->read_ev[wait_layer], 0) != cudaSuccess) return SAEM_ERR_CUDA;
     }
     if (cudaMemcpyAsync(c->slot_region + (size_t)gslot * c->slot_bytes, pinned, c->slot_bytes, cudaMemcpyHostToDevice,
@@ -447,7 +461,7 @@ int saem_cache_load(saem_ctx* c, int layer, int expert, int slot, const void* pi
 int saem_cache_evict(saem_ctx* c, int layer, int expert) {
     int s = check_le(c, layer, expert);
     if (s != SAEM_OK) return s;
-    size_t le = (size_t)layer * c->cfg.n_experts + expert;
+    size_t le = (size_t)layer * c->n_total + expert;
     if (c->slot_of[le] >= 0) {
         c->slot_owner[c->slot_of[le]] = -1;
         c->slot_of[le] = -1;
@@ -464,7 +478,7 @@ int saem_cache_evict(saem_ctx* c, int layer, int expert) {
 int saem_cache_query(saem_ctx* c, int layer, int expert, int* slot, int* ready) {
     int s = check_le(c, layer, expert);
     if (s != SAEM_OK) return s;
-    size_t le = (size_t)layer * c->cfg.n_experts + expert;
+    size_t le = (size_t)layer * c->n_total + expert;
     int gs = c->slot_of[le] >= 0 ? c->slot_of[le] : c->temp_of[le];
     if (slot) *slot = gs;
     if (ready) {
@@ -481,7 +495,7 @@ int saem_cache_query(saem_ctx* c, int layer, int expert, int* slot, int* ready) 
 int saem_cache_wait(saem_ctx* c, int layer, int expert, void* consumer) {
     int s = check_le(c, layer, expert);
     if (s != SAEM_OK) return s;
-    size_t le = (size_t)layer * c->cfg.n_experts + expert;
+    size_t le = (size_t)layer * c->n_total + expert;
     int gs = c->slot_of[le] >= 0 ? c->slot_of[le] : c->temp_of[le];
     if (gs < 0 || !c->ev_recorded[gs]) return SAEM_ERR_NOT_RESIDENT;
     CUDA_TRY(cudaStreamWaitEvent((cudaStream_t)consumer, c->ready_ev[gs], 0));

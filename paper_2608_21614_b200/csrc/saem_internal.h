@@ -66,10 +66,10 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
                          cudaStream_t st);
 // Returns the number of kernels launched (1 or 2) in *n_launch.
-cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, int k, int d, int32_t* counts,
+cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, int S, int k, int d, int32_t* counts,
                           int32_t* offsets, int32_t* perm, int32_t* inv_perm, uint16_t* x_packed, int* status,
                           int n_sm, cudaStream_t st, int* n_launch);
-cudaError_t launch_combine(const float* y, const int32_t* inv_perm, const float* w, int T, int k, int d,
+cudaError_t launch_combine(const float* y, const int32_t* inv_perm, const float* w, int T, int k, int S, int d,
                            const float* shared_y, void* out, int out_bf16, cudaStream_t st);
 
 struct FfnArgs {
@@ -105,6 +105,7 @@ struct saem_ctx {
     uint8_t* ws;
     saem::WorkspaceLayout lay;
     int n_fixed_slots;
+    int n_total;             // routed + shared experts per layer
     // residency: fixed slot per (layer, expert), -1 none; temp binding per (layer, expert), -1 none
     int32_t* slot_of;        // [L*E] global slot index
     int32_t* temp_of;        // [L*E] global slot index of a temporary binding
@@ -115,6 +116,8 @@ struct saem_ctx {
     cudaEvent_t* read_ev;    // [L] recorded on the compute stream after each FFN of that layer
     uint8_t* read_recorded;  // [L]
     int32_t* temp_last_layer;  // [temp_slots] layer whose FFN may still be reading the slot, -1 none
+    cudaStream_t* last_stream; // [L] stream of the layer's most recent FFN
+    uint8_t* ffn_seen;         // [L] 1 once an FFN of the layer has been enqueued
     int next_temp;
     bool dynamic_residency;  // fewer fixed slots than experts, or temporary slots exist: events are kept
     long long launches;

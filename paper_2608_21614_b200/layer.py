@@ -17,28 +17,37 @@ from . import binding as B
 class MoELayer:
     def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, max_tokens: int, d_ff_shared: int = 0,
                  n_layers: int = 1, slots_per_layer: Optional[int] = None, temp_slots: int = 0, renorm: int = 1,
-                 out_dtype: int = B.SAEM_OUT_F32, ffn_path: int = B.SAEM_FFN_AUTO, device: str = "cuda:0"):
+                 out_dtype: int = B.SAEM_OUT_F32, ffn_path: int = B.SAEM_FFN_AUTO, device: str = "cuda:0",
+                 merge_shared: bool = True):
         self.device = torch.device(device)
         self.d, self.f, self.E, self.k, self.max_T = d_model, d_ff, n_experts, top_k, max_tokens
-        self.cfg = B.make_config(d_model, d_ff, n_experts, top_k, max_tokens, n_layers, slots_per_layer, temp_slots,
-                                 renorm, out_dtype, ffn_path)
+        # A shared expert whose width is a multiple of d_ff runs inside the layer's grouped launch
+        # as S always-on experts of width d_ff; any other width gets a context of its own.
+        S = d_ff_shared // d_ff if (merge_shared and d_ff_shared and d_ff_shared % d_ff == 0) else 0
+        if S > 16 or n_experts + S > B.SAEM_MAX_EXPERTS:
+            S = 0
+        self.S = S
+        self.cfg = B.make_config(d_model, d_ff, n_experts, top_k, max_tokens, n_layers,
+                                 None if slots_per_layer is None else slots_per_layer + S, temp_slots, renorm,
+                                 out_dtype, ffn_path, n_shared=S)
         self.ctx = B.Context(self.cfg, device)
         self.shared: Optional[B.Context] = None
-        if d_ff_shared:
+        if d_ff_shared and S == 0:
             scfg = B.make_config(d_model, d_ff_shared, 1, 1, max_tokens, n_layers, 1, 0, 1, B.SAEM_OUT_F32, ffn_path)
             self.shared = B.Context(scfg, device)
         self.copy_stream = torch.cuda.Stream(device=self.device)
         P = max_tokens * top_k
+        R = max_tokens * (top_k + S)                 # packed rows: pairs, then T rows per in-layer shared expert
         dev = self.device
         self.topk_idx = torch.empty((max_tokens, top_k), dtype=torch.int32, device=dev)
         self.topk_w = torch.empty((max_tokens, top_k), dtype=torch.float32, device=dev)
-        self.counts = torch.empty(n_experts, dtype=torch.int32, device=dev)
-        self.offsets = torch.empty(n_experts + 1, dtype=torch.int32, device=dev)
+        self.counts = torch.empty(n_experts + S, dtype=torch.int32, device=dev)
+        self.offsets = torch.empty(n_experts + S + 1, dtype=torch.int32, device=dev)
         self.perm = torch.empty(P, dtype=torch.int32, device=dev)
         self.inv_perm = torch.empty(P, dtype=torch.int32, device=dev)
-        self.x_packed = torch.empty((P, d_model), dtype=torch.uint16, device=dev)
-        self.y_packed = torch.empty((P, d_model), dtype=torch.float32, device=dev)
-        self.shared_y = torch.empty((max_tokens, d_model), dtype=torch.float32, device=dev) if d_ff_shared else None
+        self.x_packed = torch.empty((R, d_model), dtype=torch.uint16, device=dev)
+        self.y_packed = torch.empty((R, d_model), dtype=torch.float32, device=dev)
+        self.shared_y = torch.empty((max_tokens, d_model), dtype=torch.float32, device=dev) if self.shared else None
         self.out = torch.empty((max_tokens, d_model),
                                dtype=torch.float32 if out_dtype == B.SAEM_OUT_F32 else torch.uint16, device=dev)
         self._pinned = []          # keep packed host buffers alive while copies may be in flight
@@ -60,7 +69,14 @@ class MoELayer:
                 cache[key] = self.ctx.pack(gate[e], up[e], down[e])
                 self._pinned.append(cache[key])
             B.saem_cache_load(self.ctx.handle, layer, e, e, cache[key], self.copy_stream)
-        if shared is not None:
+        if shared is not None and self.S:
+            sg, su, sd = shared
+            for s in range(self.S):                  # hidden units [s f, (s+1) f) of the wide shared expert
+                rows = slice(s * self.f, (s + 1) * self.f)
+                packed = self.ctx.pack(sg[rows], su[rows], np.ascontiguousarray(sd[:, rows]))
+                self._pinned.append(packed)
+                B.saem_cache_load(self.ctx.handle, layer, self.E + s, self.E + s, packed, self.copy_stream)
+        elif shared is not None:
             packed = self.shared.pack(*shared)
             self._pinned.append(packed)
             B.saem_cache_load(self.shared.handle, layer, 0, 0, packed, self.copy_stream)
@@ -78,11 +94,18 @@ class MoELayer:
                       self.x_packed, stream)
 
     def expert_ffn(self, T: int, layer: int = 0, subset=None, stream=None):
-        B.saem_expert_ffn(self.ctx.handle, layer, self.x_packed, self.offsets, T * self.k, subset, self.y_packed,
-                          stream)
+        B.saem_expert_ffn(self.ctx.handle, layer, self.x_packed, self.offsets, T * (self.k + self.S), subset,
+                          self.y_packed, stream)
 
     def shared_ffn(self, x: torch.Tensor, T: int, layer: int = 0, stream=None):
         B.saem_expert_ffn(self.shared.handle, layer, x, None, T, None, self.shared_y, stream)
+
+    def shared_rows(self, T: int) -> torch.Tensor:
+        """Output of the shared expert(s) for the last step: [T, d] fp32 (sums the in-layer parts)."""
+        if self.S:
+            P = T * self.k
+            return self.y_packed[P:P + self.S * T].view(self.S, T, self.d).sum(0)
+        return self.shared_y[:T]
 
     def combine(self, T: int, stream=None):
         B.saem_combine(self.ctx.handle, self.y_packed, self.inv_perm, self.topk_w, T, self.shared_y, self.out, stream)

@@ -55,13 +55,18 @@ def run_stepwise_and_compare(layer, li, oracle, ref=None):
     assert layer.device_status() == 0
     assert np.array_equal(host(layer.topk_idx[:T]), ref["topk_idx"]), "topk_idx"
     assert np.abs(host(layer.topk_w[:T]).astype(np.float64) - ref["topk_w"]).max() <= W_TOL, "topk_w"
-    assert np.array_equal(host(layer.counts), ref["counts"]), "counts"
-    assert np.array_equal(host(layer.offsets), ref["offsets"]), "offsets"
+    E = c.n_experts
+    assert np.array_equal(host(layer.counts)[:E], ref["counts"]), "counts"
+    assert np.array_equal(host(layer.offsets)[:E + 1], ref["offsets"]), "offsets"
+    if layer.S:                                      # in-layer shared experts: one segment of T rows each
+        assert np.all(host(layer.counts)[E:] == T), "shared counts"
+        assert np.array_equal(host(layer.offsets)[E:], P + T * np.arange(layer.S + 1)), "shared offsets"
+        assert np.array_equal(host(layer.x_packed[P:P + layer.S * T]), np.tile(li.x, (layer.S, 1))), "shared x rows"
     assert np.array_equal(host(layer.perm[:P]), ref["perm"]), "perm"
     assert np.array_equal(host(layer.inv_perm[:P]), ref["inv_perm"]), "inv_perm"
     assert np.array_equal(host(layer.x_packed[:P]), ref["x_packed"]), "x_packed"
     stats = {"y_packed": assert_close(host(layer.y_packed[:P]), ref["y_packed"], "y_packed")}
     if li.shared is not None:
-        stats["shared_y"] = assert_close(host(layer.shared_y[:T]), ref["shared_y"], "shared_y")
+        stats["shared_y"] = assert_close(host(layer.shared_rows(T)), ref["shared_y"], "shared_y")
     stats["out"] = assert_close(host(out), ref["out"], "out")
     return ref, stats

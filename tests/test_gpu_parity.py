@@ -154,12 +154,18 @@ def test_repack_skew_and_paper_example(oracle, B):
         ctx.close()
 
 
-def test_step_calls_agree_bit_for_bit(oracle):
-    """saem_moe_step and saem_moe_step_host give the bits of the four separate calls."""
+@pytest.mark.parametrize("fs,merge", [(256, True), (768, True), (768, False)],
+                         ids=["own-context", "in-layer", "in-layer-width-forced-separate"])
+def test_step_calls_agree_bit_for_bit(oracle, fs, merge):
+    """saem_moe_step and saem_moe_step_host give the bits of the four separate calls, with the
+    shared expert in a context of its own (width not a multiple of d_ff, or forced) and inside
+    the layer's grouped launch (width 2 x d_ff)."""
     g = _g()
-    cfg = gen.LayerConfig("t", 256, 384, 12, 3, 20, 256, "zipf", 1.1, seed=5)
+    cfg = gen.LayerConfig("t", 256, 384, 12, 3, 20, fs, "zipf", 1.1, seed=5)
     li = gen.layer_inputs(cfg)
-    layer = g.make_layer(li, TENSOR)
+    layer = g.make_layer(li, TENSOR, merge_shared=merge)
+    assert (layer.S == 2) == (fs == 768 and merge)
+    g.run_stepwise_and_compare(layer, li, oracle)
     logits, x = g.dev(li.logits), g.dev(li.x)
     ref_out = layer.step(logits, x, cfg.tokens).clone()
     out2 = torch.empty_like(ref_out)
