@@ -57,6 +57,7 @@ def layer_config(name: str, tokens: Optional[int] = None, routing: Optional[str]
     c1 tiny; c2 Mixtral-8x7B-shaped decode; c3 fine-grained (64 routed top-6 + 2 shared);
     c4 Qwen-MoE-shaped (60 routed top-4 + one wide shared expert); c5 the Mixtral-shaped
     32-layer stack (per-layer shape only; the trace comes from :func:`stage_trace`).
+    "qwen3" / "ernie": layers shaped like the paper's two models (Qwen3-30B-A3B, ERNIE-4.5-21B-A3B).
     """
     table = {
         "c1": LayerConfig("c1", 512, 1024, 8, 2, 64, 0, "normal"),
@@ -64,6 +65,10 @@ def layer_config(name: str, tokens: Optional[int] = None, routing: Optional[str]
         "c3": LayerConfig("c3", 2048, 1408, 64, 6, 32, 2 * 1408, "zipf", 1.1),
         "c4": LayerConfig("c4", 2048, 1408, 60, 4, 8, 5632, "zipf", 1.1),
         "c5": LayerConfig("c5", 4096, 14336, 8, 2, 1, 0, "zipf", 1.2, 0, 32),
+        # the paper's two evaluated models (model table): 128 routed experts top-8, no shared expert,
+        # 4.72 M parameters per expert; 64 routed top-6 + 2 shared experts
+        "qwen3": LayerConfig("qwen3", 2048, 768, 128, 8, 8, 0, "zipf", 1.1, 0, 48),
+        "ernie": LayerConfig("ernie", 2560, 1536, 64, 6, 8, 2 * 1536, "zipf", 1.1, 0, 28),
     }
     cfg = table[name]
     if tokens is not None:

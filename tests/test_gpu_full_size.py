@@ -22,7 +22,9 @@ def test_c2_mixtral_shaped_decode_full(oracle):
 
 
 @pytest.mark.parametrize("name,T,routing", [("c3", 32, "zipf"), ("c4", 1, "zipf"), ("c4", 8, "zipf"),
-                                            ("c4", 8, "uniform"), ("c4", 64, "zipf"), ("c4", 64, "uniform")])
+                                            ("c4", 8, "uniform"), ("c4", 64, "zipf"), ("c4", 64, "uniform"),
+                                            ("qwen3", 1, "zipf"), ("qwen3", 8, "zipf"), ("qwen3", 200, "zipf"),
+                                            ("ernie", 8, "zipf")])
 def test_fine_grained_decode_full(oracle, name, T, routing):
     import gpu_util as g
     li = gen.layer_inputs(gen.layer_config(name, tokens=T, routing=routing))
