@@ -28,7 +28,8 @@ constexpr int kEpiThreads = 256;
 constexpr int kGateUpMaxTile = 128;           // widest token tile of the gate/up phase (two accumulator sets fit TMEM)
 constexpr int kMaxStages = 8;
 constexpr int kDynSmemMax = 220 * 1024;
-constexpr long long kSplitBelowItemsPerCta = 6;   // split items across CTAs only below this many items per CTA
+constexpr long long kSplitBelowItemsPerCta = 6;
+constexpr long long kMinChunksPerCta = 6;      // below this many k-chunks per CTA, use fewer CTAs   // split items across CTAs only below this many items per CTA
 
 // --------------------------------------------------------------------------------------- the plan
 struct Plan {
@@ -191,10 +192,15 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     // the same number of bytes; with many items per CTA whole items are dealt out instead and no
     // partial tiles are needed.
     const long long total_chunks = (long long)plan.total_items * KC;
-    const long long G = gridDim.x;
+    // Tiny launches use fewer CTAs, so that no item is cut into dozens of slivers whose partial
+    // tiles would then have to be added up one after the other.
+    long long G = gridDim.x;
+    if (total_chunks < G * kMinChunksPerCta) G = total_chunks / kMinChunksPerCta > 0 ? total_chunks / kMinChunksPerCta : 1;
+    const long long my_cta = blockIdx.x < G ? blockIdx.x : G - 1;     // surplus CTAs get an empty range below
     const bool split_k = (long long)plan.total_items < kSplitBelowItemsPerCta * G;
-    const long long c0 = split_k ? total_chunks * blockIdx.x / G : (long long)blockIdx.x;
-    const long long c1 = split_k ? total_chunks * (blockIdx.x + 1) / G : (long long)plan.total_items;
+    long long c0 = split_k ? total_chunks * my_cta / G : my_cta;
+    long long c1 = split_k ? total_chunks * (my_cta + 1) / G : (long long)plan.total_items;
+    if (blockIdx.x >= G) c1 = c0;
     const long long walk_stride = split_k ? 0 : G;
     volatile int* abort_p = &abort_flag;
 
