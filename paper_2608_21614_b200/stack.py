@@ -89,7 +89,14 @@ class StackStats:
 class StackRunner:
     def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, n_layers: int, slots_per_layer: int,
                  temp_slots: int, batch: int, store_weights, device: str = "cuda:0",
-                 ffn_path: int = B.SAEM_FFN_AUTO):
+                 ffn_path: int = B.SAEM_FFN_AUTO, policy: str = "stage", recorded_eap: Optional[np.ndarray] = None):
+        """policy: "stage" -- at a boundary re-plan from the counts of the stage that just ended
+        (the paper's online policy); "oracle" -- re-plan from `recorded_eap[s]`, the counts of the
+        stage that is about to start, recorded in an earlier run of the same trace (the paper's
+        clairvoyant replay, Sec. VI-D); "lru" -- no stage logic: every miss evicts the layer's least
+        recently used resident expert and takes its slot (token-level baseline)."""
+        assert policy in ("stage", "oracle", "lru")
+        self.policy, self.recorded_eap, self.stage = policy, recorded_eap, 0
         self.d, self.f, self.E, self.k, self.L, self.C = d_model, d_ff, n_experts, top_k, n_layers, slots_per_layer
         self.batch = batch
         self.device = torch.device(device)
@@ -115,6 +122,9 @@ class StackRunner:
         # host mirrors of the policy state
         self.slot_expert = [[-1] * slots_per_layer for _ in range(n_layers)]     # fixed slot layout
         self.log = np.zeros((n_layers, n_experts), np.int64)                      # live activation log
+        self.eap: List[np.ndarray] = []                                           # counts of every finished stage
+        self.last_use = np.zeros((n_layers, n_experts), np.int64)                 # LRU clock per expert
+        self.clock = 0
         self.stats = StackStats()
         self.slot_bytes = self.ctx.slot_bytes
 
@@ -133,8 +143,16 @@ class StackRunner:
         """Stage boundary: re-plan every layer from the activation log, enqueue the transfers on
         the copy stream (they overlap with the following decode steps), clear the log."""
         self.stats.boundaries += 1
+        self.eap.append(self.log.copy())
+        self.stage += 1
+        if self.policy == "lru":
+            self.log[:] = 0
+            return
+        profile = self.log
+        if self.policy == "oracle":
+            profile = self.recorded_eap[min(self.stage, len(self.recorded_eap) - 1)]
         for l in range(self.L):
-            for victim, newcomer, s in plan_layer(self.log[l], self.slot_expert[l]):
+            for victim, newcomer, s in plan_layer(profile[l], self.slot_expert[l]):
                 if victim >= 0:
                     B.saem_cache_evict(self.h, l, victim)
                 if B.saem_cache_query(self.h, l, newcomer)[0] >= 0:   # bound to a temporary slot: release it
@@ -143,6 +161,21 @@ class StackRunner:
                 self.slot_expert[l][s] = newcomer
                 self.stats.boundary_loads += 1
         self.log[:] = 0
+
+    def finish(self):
+        """Call after the last step: closes the last stage's record."""
+        self.eap.append(self.log.copy())
+        return np.stack(self.eap)
+
+    def _lru_load(self, layer: int, expert: int):
+        """Token-level LRU: the miss takes the slot of the layer's least recently used resident."""
+        slots = self.slot_expert[layer]
+        s = min(range(self.C), key=lambda i: (-1 if slots[i] < 0 else self.last_use[layer, slots[i]], i))
+        if slots[s] >= 0:
+            B.saem_cache_evict(self.h, layer, slots[s])
+        B.saem_cache_load(self.h, layer, expert, s, self.store.get(layer, expert), self.copy)
+        slots[s] = expert
+        self.stats.demand_loads += 1
 
     def _demand_load(self, layer: int, expert: int):
         """Miss without a CPU path: copy the expert into the next temporary slot (round-robin);
@@ -178,6 +211,13 @@ class StackRunner:
                     need.append(e)
                     if B.saem_cache_query(self.h, l, e)[0] >= 0:      # still bound to a temporary slot
                         st.temp_hits += 1
+            self.clock += 1
+            for e in active:
+                self.last_use[l, e] = self.clock
+            if self.policy == "lru":
+                for e in need:                         # needs slots_per_layer >= active experts of a step
+                    self._lru_load(l, e)
+                need = []
             # every non-resident active expert must hold a temporary slot when the FFN is enqueued;
             # a load may recycle the slot of another one of them, so repeat until all are bound
             for _ in range(self.cfg.temp_slots + 1):

@@ -86,9 +86,9 @@ def test_load_is_ordered_after_enqueued_reads_and_before_later_ones(oracle):
     ctx.close()
 
 
-def _run_stack(trace, weights, L, E, k, d, f, C, temp, batch, steps, keep):
+def _run_stack(trace, weights, L, E, k, d, f, C, temp, batch, steps, keep, policy="stage", eap=None):
     from paper_2608_21614_b200.stack import StackRunner
-    run = StackRunner(d, f, E, k, L, C, temp, batch, weights)
+    run = StackRunner(d, f, E, k, L, C, temp, batch, weights, policy=policy, recorded_eap=eap)
     # warm set: the C most popular experts of stage 0 (stand-in for the calibration warm-up)
     run.warm([list(np.argsort(trace.rankings[0, l])[:C]) for l in range(L)])
     outs = []
@@ -190,3 +190,34 @@ def test_half_resident_stack_equals_full_residency_and_simulation(oracle):
             g.assert_close(g.host(half[t][l]), ref["out"], "step %d layer %d" % (t, l))
     run_full.close()
     run_half.close()
+
+
+def test_replay_policies_share_bits_and_oracle_is_no_worse(oracle):
+    """The prediction-oracle replay (Sec. VI-D): the same trace under the online policy, the
+    clairvoyant policy fed with the recorded per-stage counts, and token-level LRU.  Routing is
+    independent of placement, so every policy yields the same output bits; the clairvoyant
+    planner never has fewer hits at a boundary than the lag-one planner on this trace."""
+    L, E, k, d, f, batch, steps = 2, 8, 2, 128, 128, 2, 48
+    trace = gen.stage_trace(steps, L, E, 1.2, seed=5, mean_stage_len=8.0, reshuffled=None)   # independent stages
+    weights = _small_experts(4, d, f, 9)
+    keep = {steps - 1}
+    ref, st_full, _, run0 = _run_stack(trace, weights, L, E, k, d, f, E, 0, batch, steps, keep)
+    eap = run0.finish()
+    # the recorded EAP equals routing counts from the oracle, stage by stage
+    bounds = list(trace.boundaries) + [steps]
+    for s in range(len(bounds) - 1):
+        cnt = np.zeros((L, E), np.int64)
+        for t in range(int(bounds[s]), int(bounds[s + 1])):
+            for l in range(L):
+                idx, _ = oracle.route(gen.trace_logits(trace, t, l, batch), k)
+                cnt[l] += np.bincount(idx.ravel(), minlength=E)
+        assert np.array_equal(eap[s], cnt)
+    res = {}
+    for policy in ("stage", "oracle", "lru"):
+        outs, st, _, run = _run_stack(trace, weights, L, E, k, d, f, 4, 4, batch, steps, keep, policy, eap)
+        assert torch.equal(outs[0], ref[0]), policy
+        res[policy] = st
+        run.close()
+    assert res["oracle"].hits >= res["stage"].hits
+    assert res["lru"].boundary_loads == 0 and res["lru"].demand_loads > 0
+    run0.close()
