@@ -1,14 +1,17 @@
 // Grouped SwiGLU expert FFN over the repacked segments (Sec. IV-E: one dense batched execution
 // per expert over its contiguous rows; Sec. IV-C: weights live in fixed HBM cache slots),
-// written for sm_100a as a weight-streaming kernel:
+// written for sm_100a as a weight-streaming kernel.  It serves launches whose segments have at
+// most 64 rows (decode); larger segments go to the tensor-tiled kernels of ffn_prefill.cu.
 //
 //   * Operands are swapped: a 128-row tile of the expert's WEIGHTS is the MMA's M operand and the
-//     segment's tokens are the narrow N operand (16..256), so decode-sized segments still fill the
+//     segment's tokens are the narrow N operand (16..64), so decode-sized segments still fill the
 //     tensor core's M dimension and every weight byte is read from HBM exactly once per token tile.
 //   * Weight tiles are stored in the slot pre-swizzled (see saem_pack_expert_host), so one
 //     cp.async.bulk per stage lands a 16/32 KB tile in shared memory ready for tcgen05.mma;
 //     activation tiles come through a TMA tensor map with the same 128-byte swizzle.
-//   * One persistent CTA per SM.  The flat list of (expert, token tile, weight-row block,
+//   * Persistent CTAs, two per SM (each with half of the shared memory and only the TMEM columns
+//     it needs), so that one CTA's set-up, epilogue and split-item reduction overlap the other's
+//     streaming.  The flat list of (expert, token tile, weight-row block,
 //     k-chunk) units of the ACTIVE experts only is cut into equal contiguous ranges, one per CTA
 //     (inactive experts' weights are never touched).  A (expert, token tile, row block) item whose
 //     k-range is split across CTAs is finished by whichever contributor arrives last, which adds
@@ -28,8 +31,8 @@ constexpr int kEpiThreads = 256;
 constexpr int kGateUpMaxTile = 128;           // widest token tile of the gate/up phase (two accumulator sets fit TMEM)
 constexpr int kMaxStages = 8;
 constexpr int kDynSmemMax = 220 * 1024;
-constexpr long long kSplitBelowItemsPerCta = 6;
-constexpr long long kMinChunksPerCta = 6;      // below this many k-chunks per CTA, use fewer CTAs   // split items across CTAs only below this many items per CTA
+constexpr long long kSplitBelowItemsPerCta = 6;   // split items across CTAs only below this many items per CTA
+constexpr long long kMinChunksPerCta = 6;        // below this many k-chunks per CTA, use fewer CTAs
 
 // --------------------------------------------------------------------------------------- the plan
 struct Plan {
@@ -365,20 +368,36 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                         float sg[8], su[8];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) sg[j] = su[j] = 0.f;
-                        for (int ci = 0; ci < nc; ++ci) {
-                            const float* p = a.partials + ((size_t)s_contrib[ci] * 2 + (ci == 0 ? 1 : 0)) * a.partial_slot_floats +
-                                             (size_t)n0 * kTileRows + i;
-                            float vg[8], vu[8];
+                        // contributors several at a time: all their loads are issued before the first
+                        // sum needs a value (one L2 round trip per group of contributors, not per one);
+                        // the additions still run in ascending contributor order
+                        constexpr int CB = PHASE == 0 ? 2 : 4;     // bounded by the register budget
+                        for (int c0i = 0; c0i < nc; c0i += CB) {
+                            float vg[CB][8], vu[CB][8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) vg[j] = __ldcg(p + (size_t)j * kTileRows);
-                            if (PHASE == 0) {
+                            for (int cc = 0; cc < CB; ++cc) {
+                                const int ci = c0i + cc;
+                                if (ci < nc) {
+                                    const float* p = a.partials +
+                                                     ((size_t)s_contrib[ci] * 2 + (ci == 0 ? 1 : 0)) * a.partial_slot_floats +
+                                                     (size_t)n0 * kTileRows + i;
 #pragma unroll
-                                for (int j = 0; j < 8; ++j) vu[j] = __ldcg(p + (size_t)(n_tile + j) * kTileRows);
+                                    for (int j = 0; j < 8; ++j) vg[cc][j] = __ldcg(p + (size_t)j * kTileRows);
+                                    if (PHASE == 0) {
+#pragma unroll
+                                        for (int j = 0; j < 8; ++j) vu[cc][j] = __ldcg(p + (size_t)(n_tile + j) * kTileRows);
+                                    }
+                                }
                             }
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                sg[j] += vg[j];
-                                if (PHASE == 0) su[j] += vu[j];
+                            for (int cc = 0; cc < CB; ++cc) {
+                                if (c0i + cc < nc) {
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) {
+                                        sg[j] += vg[cc][j];
+                                        if (PHASE == 0) su[j] += vu[cc][j];
+                                    }
+                                }
                             }
                         }
 #pragma unroll

@@ -81,7 +81,7 @@ route_kernel(const float* __restrict__ logits, int T, int E, int k, int renorm, 
 
     // softmax over the winners
     float z[kPerLane];
-    float s = 0.f, n_inf = 0.f;
+    float s = 0.f;
 #pragma unroll
     for (int i = 0; i < kPerLane; ++i) {
         int j = lane + 32 * i;
@@ -89,7 +89,6 @@ route_kernel(const float* __restrict__ logits, int T, int E, int k, int renorm, 
         if (j < k) {
             if (vmax == CUDART_INF_F) {
                 z[i] = (win_v[i] == CUDART_INF_F) ? 1.f : 0.f;
-                n_inf += z[i];
             } else if (vmax == -CUDART_INF_F) {
                 z[i] = 1.f;
             } else {

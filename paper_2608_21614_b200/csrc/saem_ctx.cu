@@ -171,7 +171,7 @@ int saem_create(const saem_config* cfg, void* slot_region, size_t slot_region_by
     for (int i = 0; ok && i < cfg->n_layers; ++i)
         ok = cudaEventCreateWithFlags(&c->read_ev[i], cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaHostAlloc((void**)&c->pinned_status, sizeof(int), cudaHostAllocDefault) == cudaSuccess;
-    // status word, counters and the step buffers start at zero (h, partials need no clearing)
+    // the status word and the split-K arrival counters start at zero; nothing else needs clearing
     ok = ok && cudaMemsetAsync(c->ws + lay.status, 0, lay.h - lay.status, 0) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(0) == cudaSuccess;
     if (ok && cfg->ffn_path != SAEM_FFN_SCALAR) ok = ffn_tensor_init() == cudaSuccess;
