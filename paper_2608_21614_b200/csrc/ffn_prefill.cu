@@ -2,9 +2,8 @@
 // contraction, so it is tiled for the tensor cores rather than for bytes (Sec. IV-E: one dense
 // batched execution per expert over its contiguous rows).
 //
-//   * Item: kPfTokens (128) tokens of one expert's segment (the MMA's M operand, loaded by TMA
-//     from x_packed / h; the code also supports two M tiles per item sharing each weight stage)
-//     x 256 weight rows (the N operand: for gate/up the 128 gate rows and the 128 up
+//   * Item: 128 or 256 tokens of one expert's segment (one or two MMA M = 128 tiles that share
+//     every weight stage; loaded by TMA from x_packed / h) x 256 weight rows (the N operand: for gate/up the 128 gate rows and the 128 up
 //     rows of one f-block, which the packed slot layout stores back to back; for the down
 //     projection two adjacent 128-row d-blocks) x 64 reduction elements per pipeline stage.
 //     tcgen05.mma 128x256x16, fp32 accumulators in TMEM: 256 columns per 128-token tile, a ring
@@ -16,26 +15,27 @@
 //   * One persistent CTA per SM; whole tiles are dealt round-robin in the order (expert, weight
 //     block, token tile), so the CTAs that run at the same time share a weight block and it is
 //     fetched from HBM once and re-read from L2.  No tile is split, nothing is reduced across CTAs.
+//   * 128 or 256 tokens per item is decided per launch on the device: a stage is released only
+//     when its MMAs have completed and its refill takes about a microsecond, so with 4 x 48 KB
+//     stages of 128-token items the tensor pipe idles about a third of the time; two token tiles
+//     per 64 KB stage double the MMA work behind each refill (3 stages), which is faster whenever
+//     the launch still has several rounds of such items per SM.
 //   * Warp roles and bounded mbarrier waits as in the streaming kernel (ffn_tensor.cu).
 #include "tc_common.cuh"
 
 namespace saem {
 
 constexpr int kPfThreads = 320;            // warp 0 copies, warp 1 MMA, warps 2..9 epilogue
-// Tokens per item.  128 = one MMA tile per item and four pipeline stages; 256 = two MMA tiles that
-// share every weight stage (a third fewer bytes per flop from L2, three stages, half as many
-// items).  Measured on the fine-grained 2048-token layer, 128 is faster: with a few hundred items
-// per launch the coarser items lose more to the last, partly filled round than they gain.
-constexpr int kPfTokens = 128;
 constexpr int kPfStageW = 2 * kTileBytes;  // 256 weight rows x 64 k
-constexpr int kPfStageX = kPfTokens * 128; // 256 tokens x 64 k
-constexpr int kPfStage = kPfStageW + kPfStageX;
-constexpr int kPfStages = kPfTokens == 128 ? 4 : 3;
-constexpr int kPfSmem = kPfStages * kPfStage + 1024;
+constexpr int kPfTileX = 128 * 128;        // one 128-token tile x 64 k
+constexpr int kPfMaxStages = 4;
+constexpr int kPfSmem = 4 * (kPfStageW + kPfTileX) + 1024;   // = 3 x (32 KB + 2 x 16 KB) + 1 KB as well
+constexpr int kPfPairHalfRounds = 3;       // two tiles per item only with at least this many such items per TWO CTAs
 
 struct PfPlan {
     int n_active;
     int total_items;
+    int tpi;                // tokens per item: 128 or 256
     int slot[SAEM_MAX_EXPERTS];
     int row0[SAEM_MAX_EXPERTS];
     int rows[SAEM_MAX_EXPERTS];
@@ -53,12 +53,13 @@ __device__ __forceinline__ void pf_decode(const PfPlan& plan, int it, int& curso
     while (cursor + 1 < plan.n_active && plan.item_base[cursor + 1] <= it) ++cursor;
     o.a = cursor;
     const int local = it - plan.item_base[cursor];
-    const int m_blocks = (plan.rows[cursor] + kPfTokens - 1) / kPfTokens;
+    const int tpi = plan.tpi;
+    const int m_blocks = (plan.rows[cursor] + tpi - 1) / tpi;
     o.wb = local / m_blocks;
     o.mb = local - o.wb * m_blocks;
-    o.row_start = plan.row0[cursor] + o.mb * kPfTokens;
-    const int left = plan.rows[cursor] - o.mb * kPfTokens;
-    o.rows_here = left < kPfTokens ? left : kPfTokens;
+    o.row_start = plan.row0[cursor] + o.mb * tpi;
+    const int left = plan.rows[cursor] - o.mb * tpi;
+    o.rows_here = left < tpi ? left : tpi;
     o.n_cols = (o.wb == WB - 1) ? last_cols : 256;
     o.n_mt = o.rows_here > 128 ? 2 : 1;
 }
@@ -69,10 +70,10 @@ __global__ void __launch_bounds__(kPfThreads, 1)
 ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_constant__ CUtensorMap act_map) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ PfPlan plan;
-    __shared__ __align__(8) uint64_t bar_full[kPfStages], bar_empty[kPfStages], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ __align__(8) uint64_t bar_full[kPfMaxStages], bar_empty[kPfMaxStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
-    __shared__ int s_warp_act[kPfThreads / 32], s_warp_items[kPfThreads / 32];
+    __shared__ int s_warp_act[kPfThreads / 32], s_warp_t1[kPfThreads / 32], s_warp_t2[kPfThreads / 32];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int K = PHASE == 0 ? a.d : a.f;
@@ -84,7 +85,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int s = 0; s < kPfStages; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
+        for (int s = 0; s < kPfMaxStages; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_acc_full[s]), 1); mbar_init(smem_u32(&bar_acc_empty[s]), 8); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -110,40 +111,48 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 rows = 0;
             }
         }
-        const int my_items = rows > 0 ? ((rows + kPfTokens - 1) / kPfTokens) * WB : 0;
-        int act_inc = rows > 0 ? 1 : 0, item_inc = my_items;
+        const int t1 = rows > 0 ? (rows + 127) / 128 : 0, t2 = rows > 0 ? (rows + 255) / 256 : 0;   // 128- / 256-token tiles
+        int act_inc = rows > 0 ? 1 : 0, t1_inc = t1, t2_inc = t2;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const int na = __shfl_up_sync(0xffffffffu, act_inc, o), ni = __shfl_up_sync(0xffffffffu, item_inc, o);
-            if (lane >= o) { act_inc += na; item_inc += ni; }
+            const int na = __shfl_up_sync(0xffffffffu, act_inc, o), n1 = __shfl_up_sync(0xffffffffu, t1_inc, o),
+                      n2 = __shfl_up_sync(0xffffffffu, t2_inc, o);
+            if (lane >= o) { act_inc += na; t1_inc += n1; t2_inc += n2; }
         }
-        if (lane == 31) { s_warp_act[warp] = act_inc; s_warp_items[warp] = item_inc; }
+        if (lane == 31) { s_warp_act[warp] = act_inc; s_warp_t1[warp] = t1_inc; s_warp_t2[warp] = t2_inc; }
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        int base_act = 0, base_items = 0, tot_act = 0, tot_items = 0;
+        int base_act = 0, base_t1 = 0, base_t2 = 0, tot_act = 0, tot_t1 = 0, tot_t2 = 0;
 #pragma unroll
         for (int w = 0; w < kPfThreads / 32; ++w) {
-            if (w < warp) { base_act += s_warp_act[w]; base_items += s_warp_items[w]; }
+            if (w < warp) { base_act += s_warp_act[w]; base_t1 += s_warp_t1[w]; base_t2 += s_warp_t2[w]; }
             tot_act += s_warp_act[w];
-            tot_items += s_warp_items[w];
+            tot_t1 += s_warp_t1[w];
+            tot_t2 += s_warp_t2[w];
         }
+        // two token tiles per item when that still leaves several rounds of items per CTA and most
+        // of those items really have two tiles (every thread takes the same decision)
+        const bool pair = 2ll * tot_t2 * WB >= (long long)kPfPairHalfRounds * gridDim.x && 2 * tot_t1 >= 3 * tot_t2;
         if (rows > 0) {
             const int n = base_act + act_inc - 1;
             plan.slot[n] = tab.slot[e];
             plan.row0[n] = r0;
             plan.rows[n] = rows;
-            plan.item_base[n] = base_items + item_inc - my_items;
+            plan.item_base[n] = pair ? (base_t2 + t2_inc - t2) * WB : (base_t1 + t1_inc - t1) * WB;
         }
         if (tid == 0) {
-            plan.item_base[tot_act] = tot_items;
+            plan.item_base[tot_act] = (pair ? tot_t2 : tot_t1) * WB;
             plan.n_active = tot_act;
-            plan.total_items = tot_items;
+            plan.total_items = (pair ? tot_t2 : tot_t1) * WB;
+            plan.tpi = pair ? 256 : 128;
         }
         __syncthreads();
     }
     const uint32_t tmem_base = tmem_base_s;
     const int total_items = plan.total_items;
+    const int n_stages = plan.tpi == 128 ? 4 : 3;
+    const uint32_t stage_bytes = kPfStageW + (uint32_t)(plan.tpi / 128) * kPfTileX;
     const int G = gridDim.x;
     volatile int* abort_p = &abort_flag;
 
@@ -169,7 +178,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 if (!ok) break;
                 if (lane == 0) {
                     const uint32_t full = smem_u32(&bar_full[stage]);
-                    const uint32_t ws = smem_base + (uint32_t)stage * kPfStage;
+                    const uint32_t ws = smem_base + (uint32_t)stage * stage_bytes;
                     mbar_expect_tx(full, w_bytes + (uint32_t)n_boxes * 4096u);
                     bulk_g2s(ws, w0 + (size_t)kc * w_step, kTileBytes, full);
                     if (it.n_cols == 256) bulk_g2s(ws + kTileBytes, w1 + (size_t)kc * w_step, kTileBytes, full);
@@ -177,7 +186,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                         tma_2d(ws + kPfStageW + (uint32_t)b * 4096u, &act_map, kc * kTileK, it.row_start + b * 32, full);
                 }
                 ++issued;
-                if (++stage == kPfStages) { stage = 0; phase ^= 1u; }
+                if (++stage == n_stages) { stage = 0; phase ^= 1u; }
             }
         }
         if (!ok && issued > 0) {     // let copies already in flight land before the CTA's memory goes away
@@ -198,7 +207,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 ok = mbar_wait(smem_u32(&bar_full[stage]), phase, abort_p, a.status);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t ws = smem_base + (uint32_t)stage * kPfStage;
+                const uint32_t ws = smem_base + (uint32_t)stage * stage_bytes;
                 const uint32_t xs = ws + kPfStageW;
                 for (int t = 0; t < it.n_mt; ++t) {
                     const int ac = t == 0 ? acc0 : acc1;
@@ -211,14 +220,14 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                         const uint32_t d_tmem = tmem_base + (uint32_t)(ac * 256);
 #pragma unroll
                         for (int k4 = 0; k4 < kTileK / 16; ++k4)
-                            tc_mma_bf16(d_tmem, smem_desc_sw128(xs + t * (kPfStageX / 2) + k4 * 32),
+                            tc_mma_bf16(d_tmem, smem_desc_sw128(xs + t * kPfTileX + k4 * 32),
                                         smem_desc_sw128(ws + k4 * 32), idesc, (kc > 0 || k4 > 0) ? 1u : 0u);
                     }
                 }
                 if (!ok) break;
                 if (lane == 0) tc_commit(smem_u32(&bar_empty[stage]));
                 __syncwarp();
-                if (++stage == kPfStages) { stage = 0; phase ^= 1u; }
+                if (++stage == n_stages) { stage = 0; phase ^= 1u; }
             }
             if (!ok) break;
             if (lane == 0) {
