@@ -59,7 +59,7 @@ enum { SAEM_OUT_F32 = 0, SAEM_OUT_BF16 = 1 };
 enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2 };
 
 /*
- * Shape of one context.  d_model and d_ff must be multiples of 128; 1 <= top_k <= n_experts <=
+ * Shape of one context.  d_model and d_ff must be multiples of 128, at most 16384; 1 <= top_k <= n_experts <=
  * SAEM_MAX_EXPERTS; max_tokens * top_k <= 65535.  The slot region holds n_layers * slots_per_layer
  * fixed slots (slot s of layer l is global slot l * slots_per_layer + s) followed by temp_slots
  * temporary slots shared by all layers (Sec. VI ablation: on-demand loads through a reserved

@@ -4,8 +4,8 @@
 // decide an order.  The row gather moves 16 bytes per thread per access.
 //
 // Index phase, one CTA: warps take consecutive 32-pair chunks; within a chunk __match_any_sync
-// groups equal expert ids and a lane's rank is the number of lower lanes in its group; a
-// [chunk][expert] table of 16-bit counts is scanned down the chunks by one thread per expert;
+// groups equal expert ids and a lane's rank is the number of lower lanes in its group; an
+// [expert][chunk] table of 16-bit counts is scanned down the chunks by one warp per expert;
 // a scan over the expert totals gives the segment offsets.
 //
 // Small problems (pairs <= kFusedPairs): every CTA of the grid repeats the index phase in its own
@@ -32,6 +32,8 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
                                             int* __restrict__ status) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
     const int n_chunks = (P + 31) >> 5;
+    // table[e * n_chunks + c]: pairs of chunk c routed to expert e (expert-major, so that the scan
+    // down the chunks of one expert reads consecutive shared-memory words)
     for (int i = tid; i < n_chunks * E; i += blockDim.x) table[i] = 0;
     if (tid == 0) sm.bad = 0;
     __syncthreads();
@@ -43,18 +45,26 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
         int r = __popc(grp & ((1u << lane) - 1u));
         if (e >= 0) {
             rank[p] = (uint8_t)r;
-            if (r == 0) table[c * E + e] = (uint16_t)__popc(grp);
+            if (r == 0) table[e * n_chunks + c] = (uint16_t)__popc(grp);
         }
     }
     __syncthreads();
-    if (tid < E) {                                   // chunk counts -> exclusive running base per expert
+    // chunk counts -> exclusive running base per expert: one warp per expert, 32 chunks per step
+    for (int e = warp; e < E; e += n_warps) {
         int run = 0;
-        for (int c = 0; c < n_chunks; ++c) {
-            int v = table[c * E + tid];
-            table[c * E + tid] = (uint16_t)run;
-            run += v;
+        for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+            const int c = c0 + lane;
+            const int v = c < n_chunks ? table[e * n_chunks + c] : 0;
+            int inc = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int n = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += n;
+            }
+            if (c < n_chunks) table[e * n_chunks + c] = (uint16_t)(run + inc - v);
+            run += __shfl_sync(0xffffffffu, inc, 31);
         }
-        sm.counts[tid] = run;
+        if (lane == 0) sm.counts[e] = run;
     }
     __syncthreads();
     if (warp == 0) {                                 // exclusive scan over the expert totals
@@ -85,7 +95,7 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
     for (int p = tid; p < P; p += blockDim.x) {
         int e = idx[p];
         if (e < 0 || e >= E) { if (write_global) inv_perm[p] = -1; continue; }
-        int r = sm.offsets[e] + table[(p >> 5) * E + e] + rank[p];
+        int r = sm.offsets[e] + table[e * n_chunks + (p >> 5)] + rank[p];
         if (perm_s) perm_s[r] = p;
         if (write_global) { perm[r] = p; inv_perm[p] = r; }
     }

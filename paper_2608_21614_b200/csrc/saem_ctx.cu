@@ -15,6 +15,7 @@ static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int validate_config(const saem_config* c) {
     if (!c) return SAEM_ERR_INVALID_ARG;
     if (c->d_model <= 0 || c->d_ff <= 0 || c->d_model % 128 || c->d_ff % 128) return SAEM_ERR_SHAPE;
+    if (c->d_model > 16384 || c->d_ff > 16384) return SAEM_ERR_SHAPE;      // a split item has at most 256 k-chunks
     if (c->n_experts < 1 || c->n_experts > SAEM_MAX_EXPERTS) return SAEM_ERR_SHAPE;
     if (c->top_k < 1 || c->top_k > c->n_experts) return SAEM_ERR_SHAPE;
     if (c->max_tokens < 1 || (long long)c->max_tokens * c->top_k > 65535) return SAEM_ERR_SHAPE;
@@ -44,10 +45,9 @@ WorkspaceLayout workspace_layout(const saem_config& c) {
     L.status = take(256);
     L.counters = take(sizeof(int) * 2 * kMaxCtas);
     L.h = take(R * f * 2);
-    {   // split-K partial tiles: the larger of the two launch shapes (see launch_ffn_tensor)
+    {   // split-K partial tiles of the streaming kernels: token tiles of at most 64 rows, two slots per CTA
         size_t small_tile = (size_t)2 * (nt < 64 ? nt : 64) * kTileRows;
-        size_t a = (size_t)kMaxCtas * 2 * small_tile, b = (size_t)kMaxSms * 2 * L.partial_slot_floats;
-        L.partials = take((a > b ? a : b) * sizeof(float));
+        L.partials = take((size_t)kMaxCtas * 2 * small_tile * sizeof(float));
     }
     L.logits = take(T * (size_t)c.n_experts * 4);
     L.x = take(T * d * 2);
