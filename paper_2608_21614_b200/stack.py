@@ -89,13 +89,17 @@ class StackStats:
 class StackRunner:
     def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, n_layers: int, slots_per_layer: int,
                  temp_slots: int, batch: int, store_weights, device: str = "cuda:0",
-                 ffn_path: int = B.SAEM_FFN_AUTO, policy: str = "stage", recorded_eap: Optional[np.ndarray] = None):
+                 ffn_path: int = B.SAEM_FFN_AUTO, policy: str = "stage", recorded_eap: Optional[np.ndarray] = None,
+                 read_counts: bool = True):
         """policy: "stage" -- at a boundary re-plan from the counts of the stage that just ended
         (the paper's online policy); "oracle" -- re-plan from `recorded_eap[s]`, the counts of the
         stage that is about to start, recorded in an earlier run of the same trace (the paper's
         clairvoyant replay, Sec. VI-D); "lru" -- no stage logic: every miss evicts the layer's least
         recently used resident expert and takes its slot (token-level baseline)."""
         assert policy in ("stage", "oracle", "lru")
+        # With every expert resident nothing on the host depends on the routing; read_counts=False
+        # then skips the per-layer read-back (and with it the activation log and the hit statistics).
+        self.read_counts = read_counts or slots_per_layer < n_experts
         self.policy, self.recorded_eap, self.stage = policy, recorded_eap, 0
         self.d, self.f, self.E, self.k, self.L, self.C = d_model, d_ff, n_experts, top_k, n_layers, slots_per_layer
         self.batch = batch
@@ -194,6 +198,11 @@ class StackRunner:
             B.saem_route(self.h, logits_all[l], Bt, self.topk_idx, self.topk_w)
             B.saem_repack(self.h, self.topk_idx, x, Bt, self.counts, self.offsets, self.perm, self.inv_perm,
                           self.x_packed)
+            if not self.read_counts:
+                B.saem_expert_ffn(self.h, l, self.x_packed, self.offsets, Bt * k, None, self.y_packed)
+                B.saem_combine(self.h, self.y_packed, self.inv_perm, self.topk_w, Bt, None,
+                               self.out[l] if keep_out else self.out[0])
+                continue
             self.counts_host.copy_(self.counts, non_blocking=True)
             self.counts_ready.record(self.compute)
             self.counts_ready.synchronize()

@@ -32,6 +32,8 @@ def main():
     ap.add_argument("--independent", action="store_true", help="independent ranking per stage (stress trace)")
     ap.add_argument("--trace-steps", type=int, default=4096)
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-readback", action="store_true",
+                    help="with --ecr 1.0: do not read the routing counts back (no host sync per layer; no statistics)")
     args = ap.parse_args()
 
     cfg = gen.layer_config("c5")
@@ -41,7 +43,8 @@ def main():
                             reshuffled=None if args.independent else 3.2)
     rng = np.random.default_rng(np.random.SeedSequence([args.seed, 77]))
     weights = [gen.expert_weights(rng, d, f) for _ in range(args.distinct)]
-    run = StackRunner(d, f, E, k, L, C, args.temp_slots if C < E else 0, args.batch, weights)
+    run = StackRunner(d, f, E, k, L, C, args.temp_slots if C < E else 0, args.batch, weights,
+                      read_counts=not args.no_readback)
     run.warm([list(np.argsort(trace.rankings[0, l])[:C]) for l in range(L)])
     run.copy.synchronize()
     bounds = set(int(b) for b in trace.boundaries[1:])
