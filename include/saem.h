@@ -65,7 +65,9 @@ enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2 };
  * temporary slots shared by all layers (Sec. VI ablation: on-demand loads through a reserved
  * temporary slot).  renorm: 1 = softmax over the k selected logits (weights sum to 1), 0 = the
  * selected experts' probabilities under the softmax over all experts.  out_dtype: SAEM_OUT_*.
- * ffn_path: SAEM_FFN_AUTO picks the tensor-core kernels; SAEM_FFN_SCALAR forces the plain scalar
+ * ffn_path: SAEM_FFN_AUTO picks per call -- matrix-vector kernels when no segment can exceed 8
+ * rows, the tcgen05 weight-streaming kernels up to 64 rows, the tcgen05 tiled kernels beyond;
+ * SAEM_FFN_TENSOR always uses the tcgen05 kernels; SAEM_FFN_SCALAR forces the plain scalar
  * kernels (kept for triage).
  * n_shared (0..16, n_experts + n_shared <= SAEM_MAX_EXPERTS): always-on shared experts of the same
  * width d_ff that run INSIDE the layer's grouped launch.  They are experts n_experts ..

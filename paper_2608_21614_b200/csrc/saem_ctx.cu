@@ -315,10 +315,19 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     a.partials = (float*)(c->ws + c->lay.partials);
     a.partial_slot_floats = c->lay.partial_slot_floats;
     a.n_tile = n_tile_for(c, max_rows);
+    {
+        // max_rows = T * (top_k + n_shared): at most T * top_k routed experts and the n_shared shared ones have rows
+        int t = (max_rows + g.top_k + g.n_shared - 1) / (g.top_k + g.n_shared);
+        long long bound = (long long)t * g.top_k + g.n_shared;
+        a.max_active = bound < ES ? (int)bound : ES;
+    }
     a.n_sm = c->n_sm;
     int nl = 0;
+    const int seg_bound = max_rows < g.max_tokens ? max_rows : g.max_tokens;     // a token picks an expert once
     if (g.ffn_path == SAEM_FFN_SCALAR) {
         CUDA_TRY(launch_ffn_scalar(a, tab, st, &nl));
+    } else if (g.ffn_path == SAEM_FFN_AUTO && seg_bound <= 8) {
+        CUDA_TRY(launch_ffn_gemv(a, tab, st, &nl));
     } else {
         CUDA_TRY(launch_ffn_tensor(a, tab, st, &nl));
     }

@@ -86,10 +86,13 @@ struct FfnArgs {
     float* partials;
     size_t partial_slot_floats;
     int n_tile;                 // token tile for this launch (multiple of 16, <= 256)
+    int max_active;             // upper bound of experts with rows: min(E, T * top_k + n_shared)
     int n_sm;
 };
 cudaError_t launch_ffn_scalar(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
 cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
+// Segments of at most 8 rows (decode batches 1..8): row-split matrix-vector kernels.
+cudaError_t launch_ffn_gemv(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
 // One-time per process: resolves the driver entry point for tensor-map encoding and opts the
 // kernels into large dynamic shared memory.  Returns cudaSuccess or the failing error.
 cudaError_t ffn_tensor_init();

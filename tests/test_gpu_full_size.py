@@ -9,7 +9,7 @@ import torch
 from paper_2608_21614_b200 import inputs as gen
 
 pytestmark = pytest.mark.gpu
-TENSOR = 2
+TENSOR = 0      # SAEM_FFN_AUTO: the path bench.py times (matrix-vector / streaming / tiled tcgen05 by batch size)
 
 
 def test_c2_mixtral_shaped_decode_full(oracle):

@@ -9,7 +9,7 @@ from paper_2608_21614_b200 import inputs as gen
 
 pytestmark = pytest.mark.gpu
 
-SCALAR, TENSOR = 1, 2
+AUTO, SCALAR, TENSOR = 0, 1, 2
 
 
 @pytest.fixture(scope="module")
@@ -34,6 +34,23 @@ def test_c1_every_call(oracle, path):
     layer.step(g.dev(li.logits), g.dev(li.x), li.cfg.tokens)
     torch.cuda.synchronize()
     assert torch.equal(y1, layer.y_packed) and torch.equal(o1, layer.out)
+    layer.close()
+
+
+@pytest.mark.parametrize("T,E,k,d,f,fs", [(1, 1, 1, 128, 128, 0), (1, 60, 4, 256, 384, 256), (1, 60, 4, 256, 384, 384),
+                                          (8, 8, 8, 128, 256, 0), (5, 128, 8, 256, 128, 128), (8, 8, 2, 512, 1024, 0),
+                                          (3, 16, 2, 2048, 1408, 2816)])
+def test_tiny_batches_matrix_vector_path(oracle, T, E, k, d, f, fs):
+    """Batches of at most 8 tokens take the row-split matrix-vector kernels (ffn_path AUTO)."""
+    g = _g()
+    cfg = gen.LayerConfig("t", d, f, E, k, T, fs, "zipf", 1.1, seed=100 + T + E)
+    li = gen.layer_inputs(cfg, n_distinct_experts=min(E, 6))
+    layer = g.make_layer(li, AUTO)
+    g.run_stepwise_and_compare(layer, li, oracle)
+    y1 = layer.y_packed.clone()
+    layer.step(g.dev(li.logits), g.dev(li.x), T)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, layer.y_packed)                 # deterministic
     layer.close()
 
 
