@@ -297,3 +297,37 @@ def test_step_is_graph_capturable_and_replays_identically(oracle):
     g.assert_close(g.host(layer.out[:cfg.tokens]), ref["out"], "graph replay on new inputs")
     assert layer.device_status() == 0
     layer.close()
+
+
+def test_empty_batch_and_limits(B):
+    """T = 0 is a no-op everywhere (repack still zeroes counts and offsets); T = max_tokens works and
+    T = max_tokens + 1 is refused before anything is enqueued."""
+    g = _g()
+    E, k, d, f, maxT = 6, 2, 128, 128, 5
+    cfg = B.make_config(d, f, E, k, maxT)
+    ctx = B.Context(cfg)
+    h = ctx.handle
+    n0 = B.saem_launch_count(h)
+    counts = torch.full((E,), 7, dtype=torch.int32, device="cuda:0")
+    offsets = torch.full((E + 1,), 7, dtype=torch.int32, device="cuda:0")
+    z = torch.zeros(maxT * k * d, dtype=torch.float32, device="cuda:0")
+    zi = torch.zeros(maxT * k, dtype=torch.int32, device="cuda:0")
+    zx = torch.zeros((maxT * k, d), dtype=torch.uint16, device="cuda:0")
+    assert B.saem_route(h, z, 0, zi, z, check=False) == B.SAEM_OK
+    assert B.saem_combine(h, z, zi, z, 0, None, z, check=False) == B.SAEM_OK
+    assert B.saem_expert_ffn(h, 0, zx, offsets, 0, None, z, check=False) == B.SAEM_OK
+    assert B.saem_launch_count(h) == n0                       # nothing was launched
+    assert B.saem_repack(h, zi, zx, 0, counts, offsets, zi, zi, zx, check=False) == B.SAEM_OK
+    torch.cuda.synchronize()
+    assert counts.sum().item() == 0 and offsets.sum().item() == 0
+    for call in (lambda T: B.saem_route(h, z, T, zi, z, check=False),
+                 lambda T: B.saem_repack(h, zi, zx, T, counts, offsets, zi, zi, zx, check=False),
+                 lambda T: B.saem_combine(h, z, zi, z, T, None, z, check=False)):
+        assert call(maxT) == B.SAEM_OK
+        assert call(maxT + 1) == B.SAEM_ERR_SHAPE
+        assert call(-1) == B.SAEM_ERR_SHAPE
+    assert B.saem_expert_ffn(h, 0, zx, offsets, maxT * k + 1, None, z, check=False) == B.SAEM_ERR_SHAPE
+    assert B.saem_expert_ffn(h, 0, zx.view(-1)[1:], offsets, 2, None, z, check=False) == B.SAEM_ERR_ALIGNMENT
+    torch.cuda.synchronize()
+    assert B.saem_last_device_status(h) == 0
+    ctx.close()
