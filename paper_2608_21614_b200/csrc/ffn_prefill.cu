@@ -312,15 +312,14 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
 }
 
 // ------------------------------------------------------------------------------------------- host
-static bool g_pf_init = false;
+static bool g_pf_init[64];
 
 cudaError_t ffn_prefill_init() {
-    if (g_pf_init) return cudaSuccess;
+    if (!first_call_on_device(g_pf_init)) return cudaSuccess;
     cudaError_t e = cudaFuncSetAttribute(ffn_prefill_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(ffn_prefill_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmem);
     if (e != cudaSuccess) return e;
-    g_pf_init = true;
     return cudaSuccess;
 }
 

@@ -433,21 +433,23 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 static EncodeTiledFn g_encode = nullptr;
-static bool g_init_done = false;
+static bool g_init_done[64];
 
 cudaError_t ffn_tensor_init() {
-    if (g_init_done) return cudaSuccess;
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-    if (e != cudaSuccess) return e;
-    if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
-    g_encode = (EncodeTiledFn)fn;
+    if (!first_call_on_device(g_init_done)) return cudaSuccess;
+    cudaError_t e;
+    if (!g_encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+        g_encode = (EncodeTiledFn)fn;
+    }
     e = cudaFuncSetAttribute(ffn_tensor_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemMax);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(ffn_tensor_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemMax);
     if (e != cudaSuccess) return e;
-    g_init_done = true;
     return cudaSuccess;
 }
 
@@ -463,7 +465,7 @@ static bool make_act_map(CUtensorMap* m, const void* base, int rows, int K, int 
 }
 
 cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch) {
-    if (!g_init_done) {
+    {
         cudaError_t e = ffn_tensor_init();
         if (e != cudaSuccess) return e;
     }

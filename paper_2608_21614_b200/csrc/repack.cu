@@ -170,13 +170,12 @@ cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, i
                           int n_sm, cudaStream_t st, int* n_launch) {
     const int P = T * k, n_chunks = (P + 31) >> 5;
     size_t base = sizeof(RepackSmem) + (((size_t)n_chunks * E * 2 + 15) & ~(size_t)15);
-    static bool attr_done = false;
-    if (!attr_done) {
+    static bool attr_done[64];
+    if (first_call_on_device(attr_done)) {
         cudaError_t e = cudaFuncSetAttribute(repack_index_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(repack_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     if (P <= kFusedPairs) {
         size_t smem = base + (size_t)n_chunks * 32 * 4 + (size_t)n_chunks * 32;
