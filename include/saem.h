@@ -254,6 +254,15 @@ int saem_last_device_status(saem_ctx* ctx, int* code);
 /* Number of kernels this library has launched through `ctx` since creation (host counter). */
 long long saem_launch_count(saem_ctx* ctx);
 
+/*
+ * Self-test of the failure path of the kernels' device-side waits (no counterpart in the paper).
+ * Every wait inside the FFN kernels is bounded; this enqueues a one-CTA kernel that waits, with the
+ * same helper, on a barrier nothing will ever complete, with a limit of limit_us microseconds
+ * (1..1 000 000).  The kernel must return by itself and leave SAEM_ERR_TIMEOUT in the device status
+ * word (read it with saem_last_device_status); the context stays usable.  Nothing traps or hangs.
+ */
+int saem_selftest_bounded_wait(saem_ctx* ctx, int limit_us, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -66,6 +66,7 @@ def _load() -> C.CDLL:
         "saem_last_device_status": (i32, [vp, C.POINTER(i32)]),
         "saem_launch_count": (C.c_longlong, [vp]),
         "saem_expert_ffn_static": (i32, [vp, vp, i32, i32, i32, i32, vp, vp, vp]),
+        "saem_selftest_bounded_wait": (i32, [vp, i32, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -78,7 +79,7 @@ _lib = _load()
 EXPORTS = ("saem_version saem_status_string saem_slot_bytes saem_slot_region_bytes saem_workspace_bytes "
            "saem_create saem_destroy saem_pack_expert_host saem_route saem_repack saem_expert_ffn saem_combine "
            "saem_moe_step saem_moe_step_host saem_step_buffer saem_cache_load saem_cache_evict saem_cache_query "
-           "saem_cache_wait saem_last_device_status saem_launch_count saem_expert_ffn_static").split()
+           "saem_cache_wait saem_last_device_status saem_launch_count saem_expert_ffn_static saem_selftest_bounded_wait").split()
 
 
 def library_path() -> str:
@@ -248,6 +249,13 @@ def saem_last_device_status(ctx) -> int:
 
 def saem_launch_count(ctx) -> int:
     return int(_lib.saem_launch_count(ctx))
+
+
+def saem_selftest_bounded_wait(ctx, limit_us: int, stream=None, check=True) -> int:
+    code = _lib.saem_selftest_bounded_wait(ctx, limit_us, _stream(stream))
+    if check:
+        _check(code, "saem_selftest_bounded_wait")
+    return code
 
 
 SAEM_STATIC_SCRATCH_ELEMS = 1 << 20

@@ -428,6 +428,25 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     }
 }
 
+// One CTA waits, with the kernels' bounded wait, on an mbarrier that nothing ever completes: the
+// wait must run out after `limit_ns`, set SAEM_ERR_TIMEOUT in the status word and return normally.
+__global__ void bounded_wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, limit_ns);    // phase 0 never completes
+}
+
+cudaError_t launch_bounded_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(status, limit_ns);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------------------------------- host
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

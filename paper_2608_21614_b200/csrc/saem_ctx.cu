@@ -522,4 +522,12 @@ int saem_last_device_status(saem_ctx* c, int* code) {
 
 long long saem_launch_count(saem_ctx* c) { return c ? c->launches : 0; }
 
+int saem_selftest_bounded_wait(saem_ctx* c, int limit_us, void* stream) {
+    if (!c || limit_us < 1 || limit_us > 1000000) return SAEM_ERR_INVALID_ARG;
+    CUDA_TRY(launch_bounded_wait_selftest((int*)(c->ws + c->lay.status), (unsigned long long)limit_us * 1000ull,
+                                          (cudaStream_t)stream));
+    c->launches += 1;
+    return SAEM_OK;
+}
+
 }  // extern "C"

@@ -105,6 +105,8 @@ cudaError_t launch_ffn_gemv(const FfnArgs& a, const SlotTable& tab, cudaStream_t
 // One-time per process: resolves the driver entry point for tensor-map encoding and opts the
 // kernels into large dynamic shared memory.  Returns cudaSuccess or the failing error.
 cudaError_t ffn_tensor_init();
+// Exercises the kernels' bounded mbarrier wait: a 1-CTA kernel whose wait can only run out.
+cudaError_t launch_bounded_wait_selftest(int* status, unsigned long long limit_ns, cudaStream_t st);
 
 }  // namespace saem
 

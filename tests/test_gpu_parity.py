@@ -331,3 +331,22 @@ def test_empty_batch_and_limits(B):
     torch.cuda.synchronize()
     assert B.saem_last_device_status(h) == 0
     ctx.close()
+
+
+def test_bounded_device_wait_runs_out_and_context_survives(oracle, B):
+    """Failure detection without a GPU fault: a wait that nothing will ever satisfy gives up after
+    its limit, the kernel returns, the status word says TIMEOUT, and the same context then runs a
+    correct step."""
+    import time
+    g = _g()
+    li = gen.layer_inputs(gen.LayerConfig("t", 128, 128, 4, 2, 16, seed=1))
+    layer = g.make_layer(li, TENSOR)
+    t0 = time.perf_counter()
+    B.saem_selftest_bounded_wait(layer.ctx.handle, 20000)            # 20 ms limit
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 5.0
+    assert layer.device_status() == B.SAEM_ERR_TIMEOUT
+    assert layer.device_status() == 0
+    assert B.saem_selftest_bounded_wait(layer.ctx.handle, 0, check=False) == B.SAEM_ERR_INVALID_ARG
+    g.run_stepwise_and_compare(layer, li, oracle)
+    layer.close()
