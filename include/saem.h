@@ -139,6 +139,18 @@ int saem_pack_expert_host(const saem_config* cfg, const void* gate, const void* 
 int saem_route(saem_ctx* ctx, const float* logits, int T, int32_t* topk_idx, float* topk_w, void* stream);
 
 /*
+ * Gating with the router projection fused in: logits[t, e] = <x[t, :], w_router[e, :]> (x[T, d_model]
+ * and w_router[n_experts, d_model] bf16, dev, 16-byte aligned; fp32 accumulation), followed by the
+ * selection and weights of saem_route in the same kernel.  logits_out[T, n_experts] fp32 (dev) may
+ * be NULL.  The paper only says that a routing mechanism selects the top-k experts (Background,
+ * "Mixture-of-Experts Inference"); a linear router without bias is the reading taken.  Because the
+ * logits are rounded sums, two experts whose exact logits differ by less than the accumulation
+ * error (about 1e-5 relative) may swap ranks against an exact evaluation.
+ */
+int saem_route_fused(saem_ctx* ctx, const void* x, const void* w_router, int T, float* logits_out,
+                     int32_t* topk_idx, float* topk_w, void* stream);
+
+/*
  * Expert-aligned token repacking.  topk_idx[T, top_k] (dev) and x[T, d_model] bf16 (dev) ->
  * counts[n_experts], offsets[n_experts + 1] (exclusive scan, offsets[E] = T*top_k), perm[T*top_k]
  * (pair stored at packed row r), inv_perm[T*top_k] (packed row of pair p), x_packed[T*top_k,

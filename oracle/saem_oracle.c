@@ -34,6 +34,20 @@ static double bf16_to_double(uint16_t b) {
     return (double)f;
 }
 
+/* ---------------------------------------------------------------------------------- router logits
+ * Linear router without bias (the paper only names "a routing mechanism"; reading taken):
+ * logits[t, e] = sum_i x[t, i] * w_router[e, i], in double, from bf16 bit patterns.
+ */
+void saem_oracle_router_logits(const uint16_t* x, const uint16_t* w_router, int T, int E, int d, double* logits) {
+    for (int t = 0; t < T; ++t)
+        for (int e = 0; e < E; ++e) {
+            double a = 0.0;
+            for (int i = 0; i < d; ++i)
+                a += bf16_to_double(x[(size_t)t * d + i]) * bf16_to_double(w_router[(size_t)e * d + i]);
+            logits[(size_t)t * E + e] = a;
+        }
+}
+
 /* ------------------------------------------------------------------------------------------ route
  * Gating.  For each token: k rounds of arg-max over the experts not yet chosen, comparing
  * (value descending, then expert id ascending); NaN logits count as -inf; +0 and -0 are equal.

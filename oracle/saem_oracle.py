@@ -53,6 +53,17 @@ def _ptr_array(mats: Sequence[Optional[np.ndarray]]):
     return arr
 
 
+def router_logits(x: np.ndarray, w_router: np.ndarray) -> np.ndarray:
+    """float64 logits[T, E] of a bias-free linear router from bf16 bit patterns x[T, d], w_router[E, d]."""
+    x = np.ascontiguousarray(x, dtype=np.uint16)
+    w_router = np.ascontiguousarray(w_router, dtype=np.uint16)
+    T, d = x.shape
+    E = w_router.shape[0]
+    out = np.empty((T, E), np.float64)
+    _load().saem_oracle_router_logits(_p(x), _p(w_router), T, E, d, _p(out))
+    return out
+
+
 def route(logits: np.ndarray, k: int, renorm: bool = True):
     logits = np.ascontiguousarray(logits, dtype=np.float32)
     T, E = logits.shape

@@ -53,6 +53,7 @@ def _load() -> C.CDLL:
         "saem_destroy": (None, [vp]),
         "saem_pack_expert_host": (i32, [cfgp, vp, vp, vp, vp]),
         "saem_route": (i32, [vp, vp, i32, vp, vp, vp]),
+        "saem_route_fused": (i32, [vp, vp, vp, i32, vp, vp, vp, vp]),
         "saem_repack": (i32, [vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]),
         "saem_expert_ffn": (i32, [vp, i32, vp, vp, i32, vp, i32, vp, vp]),
         "saem_combine": (i32, [vp, vp, vp, vp, i32, vp, vp, vp]),
@@ -77,7 +78,7 @@ def _load() -> C.CDLL:
 
 _lib = _load()
 EXPORTS = ("saem_version saem_status_string saem_slot_bytes saem_slot_region_bytes saem_workspace_bytes "
-           "saem_create saem_destroy saem_pack_expert_host saem_route saem_repack saem_expert_ffn saem_combine "
+           "saem_create saem_destroy saem_pack_expert_host saem_route saem_route_fused saem_repack saem_expert_ffn saem_combine "
            "saem_moe_step saem_moe_step_host saem_step_buffer saem_cache_load saem_cache_evict saem_cache_query "
            "saem_cache_wait saem_last_device_status saem_launch_count saem_expert_ffn_static saem_selftest_bounded_wait").split()
 
@@ -162,6 +163,14 @@ def saem_route(ctx, logits, T, topk_idx, topk_w, stream=None, check=True) -> int
     code = _lib.saem_route(ctx, _ptr(logits), T, _ptr(topk_idx), _ptr(topk_w), _stream(stream))
     if check:
         _check(code, "saem_route")
+    return code
+
+
+def saem_route_fused(ctx, x, w_router, T, logits_out, topk_idx, topk_w, stream=None, check=True) -> int:
+    code = _lib.saem_route_fused(ctx, _ptr(x), _ptr(w_router), T, _ptr(logits_out), _ptr(topk_idx), _ptr(topk_w),
+                                 _stream(stream))
+    if check:
+        _check(code, "saem_route_fused")
     return code
 
 

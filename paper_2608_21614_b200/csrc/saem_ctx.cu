@@ -247,6 +247,19 @@ int saem_route(saem_ctx* c, const float* logits, int T, int32_t* idx, float* w, 
     return SAEM_OK;
 }
 
+int saem_route_fused(saem_ctx* c, const void* x, const void* w_router, int T, float* logits_out, int32_t* idx,
+                     float* w, void* stream) {
+    int s = check_T(c, T);
+    if (s != SAEM_OK) return s;
+    if (T == 0) return SAEM_OK;
+    if (!x || !w_router || !idx || !w) return SAEM_ERR_INVALID_ARG;
+    if (misaligned(x) || misaligned(w_router)) return SAEM_ERR_ALIGNMENT;
+    CUDA_TRY(launch_route_fused((const uint16_t*)x, (const uint16_t*)w_router, T, c->cfg.n_experts, c->cfg.d_model,
+                                c->cfg.top_k, c->cfg.renorm, logits_out, idx, w, (cudaStream_t)stream));
+    c->launches += 1;
+    return SAEM_OK;
+}
+
 int saem_repack(saem_ctx* c, const int32_t* idx, const void* x, int T, int32_t* counts, int32_t* offsets,
                 int32_t* perm, int32_t* inv_perm, void* x_packed, void* stream) {
     int s = check_T(c, T);

@@ -74,6 +74,8 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 // ---- kernel launchers (each returns a cudaError_t from the launch) ----
 cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, int32_t* idx, float* w,
                          cudaStream_t st);
+cudaError_t launch_route_fused(const uint16_t* x, const uint16_t* w_router, int T, int E, int d, int k, int renorm,
+                               float* logits_out, int32_t* idx, float* w, cudaStream_t st);
 // Returns the number of kernels launched (1 or 2) in *n_launch.
 cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, int S, int k, int d, int32_t* counts,
                           int32_t* offsets, int32_t* perm, int32_t* inv_perm, uint16_t* x_packed, int* status,

@@ -99,6 +99,11 @@ def activations(rng: np.random.Generator, tokens: int, d_model: int) -> np.ndarr
     return to_bf16_bits(rng.standard_normal((tokens, d_model), dtype=np.float32))
 
 
+def router_weights(rng: np.random.Generator, n_experts: int, d_model: int) -> np.ndarray:
+    """w_router[E, d] ~ N(0, 1/d) as bf16 bits: with x ~ N(0,1) the logits are about N(0,1)."""
+    return to_bf16_bits(rng.standard_normal((n_experts, d_model), dtype=np.float32) * np.float32(d_model ** -0.5))
+
+
 def zipf_popularity(ranking: np.ndarray, s: float) -> np.ndarray:
     """p(e) proportional to rank(e)^-s, where ranking[e] in 1..E."""
     p = ranking.astype(np.float64) ** (-float(s))

@@ -350,3 +350,36 @@ def test_bounded_device_wait_runs_out_and_context_survives(oracle, B):
     assert B.saem_selftest_bounded_wait(layer.ctx.handle, 0, check=False) == B.SAEM_ERR_INVALID_ARG
     g.run_stepwise_and_compare(layer, li, oracle)
     layer.close()
+
+
+@pytest.mark.parametrize("T,E,k,d", [(1, 60, 4, 2048), (16, 8, 2, 4096), (64, 128, 8, 2048), (33, 64, 6, 256)])
+def test_route_fused_with_router_projection(oracle, B, T, E, k, d):
+    """saem_route_fused: logits against the oracle's float64 router; selection and weights must be
+    exactly what saem_route gives on those logits, and equal the oracle's wherever the exact logits
+    are not within rounding distance of a tie."""
+    g = _g()
+    rng = np.random.default_rng(T * 131 + E)
+    x = gen.activations(rng, T, d)
+    wr = gen.router_weights(rng, E, d)
+    ctx = B.Context(B.make_config(d, 128, E, k, T))
+    idx = torch.empty((T, k), dtype=torch.int32, device="cuda:0")
+    w = torch.empty((T, k), dtype=torch.float32, device="cuda:0")
+    logits = torch.empty((T, E), dtype=torch.float32, device="cuda:0")
+    B.saem_route_fused(ctx.handle, g.dev(x), g.dev(wr), T, logits, idx, w)
+    idx2, w2 = torch.empty_like(idx), torch.empty_like(w)
+    B.saem_route(ctx.handle, logits, T, idx2, w2)
+    torch.cuda.synchronize()
+    assert torch.equal(idx, idx2) and torch.equal(w, w2)                 # same gate on the same logits
+    ref_logits = oracle.router_logits(x, wr)
+    assert np.abs(g.host(logits).astype(np.float64) - ref_logits).max() <= 1e-4
+    ridx, rw = oracle.route(ref_logits.astype(np.float32), k)
+    srt = -np.sort(-ref_logits, axis=1)[:, :min(k + 1, E)]
+    clear = (np.abs(np.diff(srt, axis=1)).min(axis=1) > 1e-4) if E > 1 else np.ones(T, bool)
+    assert clear.mean() >= 0.9
+    assert np.array_equal(g.host(idx)[clear], ridx[clear])
+    assert np.abs(g.host(w).astype(np.float64) - rw)[clear].max() <= 1e-5
+    # without the optional logits output
+    B.saem_route_fused(ctx.handle, g.dev(x), g.dev(wr), T, None, idx2, w2)
+    torch.cuda.synchronize()
+    assert torch.equal(idx, idx2) and torch.equal(w, w2)
+    ctx.close()

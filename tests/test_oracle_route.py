@@ -86,3 +86,16 @@ def test_uniform_routing_frequency(oracle):
     freq = np.bincount(idx.ravel(), minlength=E) / T
     assert abs(freq.mean() - k / E) < 1e-12
     assert np.all(np.abs(freq - 0.0625) < 6 * np.sqrt(0.0625 * 0.9375 / T))
+
+
+def test_router_logits_equal_library_matmul(oracle):
+    from paper_2608_21614_b200 import inputs as gen
+    rng = np.random.default_rng(21)
+    x = gen.activations(rng, 9, 192)
+    w = gen.router_weights(rng, 13, 192)
+    got = oracle.router_logits(x, w)
+    ref = gen.bf16_bits_to_f32(x).astype(np.float64) @ gen.bf16_bits_to_f32(w).astype(np.float64).T
+    assert got.shape == (9, 13) and np.allclose(got, ref, rtol=0, atol=1e-12)
+    assert 0.5 < got.std() < 1.5
+    onehot = gen.to_bf16_bits(np.eye(4, 192, dtype=np.float32))          # x_t = e_t picks column t of W
+    assert np.array_equal(oracle.router_logits(onehot, w), gen.bf16_bits_to_f32(w)[:, :4].T.astype(np.float64))
