@@ -157,6 +157,9 @@ int saem_route_fused(saem_ctx* ctx, const void* x, const void* w_router, int T, 
  * d_model] bf16 = x[perm[r] / top_k].  Segments are in ascending expert id and keep ascending pair
  * id inside (a stable counting sort), so the permutation is unique.  An index outside
  * [0, n_experts) sets the device status word and the pair is dropped from every output.
+ * With config.n_shared = S > 0 the outputs grow: counts[n_experts + S], offsets[n_experts + S + 1],
+ * x_packed[T*(top_k + S), d_model]; shared expert s owns rows [T*top_k + s*T, T*top_k + (s+1)*T),
+ * a copy of x, and offsets[n_experts] is T*top_k.
  */
 int saem_repack(saem_ctx* ctx, const int32_t* topk_idx, const void* x, int T, int32_t* counts,
                 int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* x_packed, void* stream);
@@ -166,8 +169,8 @@ int saem_repack(saem_ctx* ctx, const int32_t* topk_idx, const void* x, int T, in
  * x_packed (dev, bf16): y_packed[r] = Wd_e * ( silu(Wg_e * x_r) .* (Wu_e * x_r) ), fp32
  * accumulation, hidden activations rounded to bf16 in the context's workspace, y_packed[max_rows,
  * d_model] fp32 (dev).  Weights come from the slots that `layer`'s residency map (or a temporary
- * slot) gives.  offsets (dev) is read on the device only; max_rows bounds offsets[n_experts] and
- * must not exceed max_tokens * top_k.  offsets may be NULL only when n_experts == 1: the single
+ * slot) gives.  offsets (dev, n_experts + n_shared + 1 entries) is read on the device only;
+ * max_rows bounds its last entry and must not exceed max_tokens * (top_k + n_shared).  offsets may be NULL only when n_experts == 1: the single
  * segment is then rows [0, max_rows) (used for always-on shared experts, whose input is x itself).
  *   expert_subset (host, may be NULL): run only these experts (rows of the others are left
  *   untouched).  With a subset, an expert that has no slot returns NOT_RESIDENT before any
@@ -181,7 +184,8 @@ int saem_expert_ffn(saem_ctx* ctx, int layer, const void* x_packed, const int32_
 
 /*
  * Weighted merge: out[t] = sum_{j = 0..top_k-1, in that order} topk_w[t, j] *
- * y_packed[inv_perm[t*top_k + j]] (+ shared_y[t] if not NULL, fp32 [T, d_model], added last).
+ * y_packed[inv_perm[t*top_k + j]] (+ the rows y_packed[T*top_k + s*T + t] of the config.n_shared
+ * in-layer shared experts, weight 1) (+ shared_y[t] if not NULL, fp32 [T, d_model], added last).
  * Gather-based, no atomics: two runs give identical bits.  out[T, d_model] fp32 or bf16 per
  * config.out_dtype.
  */
@@ -192,7 +196,8 @@ int saem_combine(saem_ctx* ctx, const float* y_packed, const int32_t* inv_perm, 
  * The whole layer step on device buffers: route -> repack -> expert FFN -> [shared expert FFN via
  * shared_ctx over x itself] -> combine, enqueued on `stream`, intermediates in ctx's workspace.
  * shared_ctx (may be NULL) is a context with n_experts = top_k = 1 whose layer `layer` slot 0
- * holds the always-on shared expert (two shared experts of width f are packed as one of width 2f).
+ * holds an always-on shared expert whose width is not a multiple of d_ff (otherwise use
+ * config.n_shared and pass NULL).
  * logits[T, E] fp32, x[T, d] bf16, out[T, d] (all dev).
  */
 int saem_moe_step(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const float* logits, const void* x, int T,
