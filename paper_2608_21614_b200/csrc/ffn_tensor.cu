@@ -136,10 +136,16 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(tmem_cols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // Everything below reads what the preceding kernels of the stream wrote (offsets, x_packed, h).
-    // Under programmatic dependent launch this kernel may have started before they finished.
-    pdl_wait();
-    pdl_launch_dependents();
+    // Under programmatic dependent launch this kernel may have started before the preceding kernels
+    // of the stream finished.  The gate/up kernel reads what its predecessor (the repack) wrote right
+    // away (offsets), so it waits here.  The down kernel's predecessor is the gate/up kernel, which
+    // has passed this very wait before it let dependents launch: the repack's outputs are final, so
+    // the down kernel may build its plan and even start loading WEIGHTS (which no kernel writes)
+    // before it waits for h; see the producer.
+    if (PHASE == 0) {
+        pdl_wait();
+        pdl_launch_dependents();
+    }
 
     // ---- plan: active experts of this launch, in ascending id (one thread per expert) ----
     {
@@ -206,6 +212,10 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
     if (blockIdx.x >= G) c1 = c0;
     const long long walk_stride = split_k ? 0 : G;
     volatile int* abort_p = &abort_flag;
+    if (PHASE == 1 && warp != 0) {
+        pdl_wait();
+        pdl_launch_dependents();
+    }
 
     if (warp == 0) {
         // =============================== producer ===============================
@@ -215,20 +225,46 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
         uint32_t phase = 0;
         bool ok = true;
         int issued = 0;
+        int pre = 0;                 // stages whose weights went out before the dependency wait (down kernel)
+        const size_t w_region = PHASE == 0 ? 0 : (size_t)2 * a.d * a.f * 2;
+        if (PHASE == 1) {
+            // weights of the first stages: they do not depend on the gate/up kernel
+            ItemWalker early(&plan, c0, c1, walk_stride, KC, RB, n_tile);
+            Item ei;
+            while (pre < n_stages && early.next(ei)) {
+                const uint8_t* wsrc = a.slot_region + (size_t)plan.slot[ei.a] * a.slot_bytes + w_region +
+                                      (size_t)ei.rb * KC * W_BYTES;
+                const int nb = (ei.rows_here + box_rows - 1) / box_rows;
+                for (int kc = ei.kc_begin; kc < ei.kc_end && pre < n_stages; ++kc, ++pre) {
+                    if (lane == 0) {
+                        const uint32_t full = smem_u32(&bar_full[pre]);
+                        mbar_expect_tx(full, W_BYTES + (uint32_t)(nb * box_rows) * 128u);
+                        bulk_g2s(smem_base + (uint32_t)pre * stage_bytes, wsrc + (size_t)kc * W_BYTES, kTileBytes, full);
+                    }
+                }
+            }
+            pdl_wait();              // h is complete from here on
+            pdl_launch_dependents();
+        }
         while (ok && walk.next(it)) {
             const uint8_t* slot = a.slot_region + (size_t)plan.slot[it.a] * a.slot_bytes;
-            const uint8_t* wbase = slot + (PHASE == 0 ? 0 : (size_t)2 * a.d * a.f * 2) + (size_t)it.rb * KC * W_BYTES;
+            const uint8_t* wbase = slot + w_region + (size_t)it.rb * KC * W_BYTES;
             const int n_boxes = (it.rows_here + box_rows - 1) / box_rows;
             for (int kc = it.kc_begin; kc < it.kc_end; ++kc) {
-                ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, a.status);
-                if (!ok) break;
+                const bool early_w = issued < pre;          // this stage's weights are already on their way
+                if (!early_w) {
+                    ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, a.status);
+                    if (!ok) break;
+                }
                 if (lane == 0) {
                     const uint32_t full = smem_u32(&bar_full[stage]);
                     const uint32_t ws = smem_base + (uint32_t)stage * stage_bytes;
-                    mbar_expect_tx(full, W_BYTES + (uint32_t)(n_boxes * box_rows) * 128u);
-                    const uint8_t* src = wbase + (size_t)kc * W_BYTES;
-                    bulk_g2s(ws, src, kTileBytes, full);
-                    if (PHASE == 0) bulk_g2s(ws + kTileBytes, src + kTileBytes, kTileBytes, full);
+                    if (!early_w) {
+                        mbar_expect_tx(full, W_BYTES + (uint32_t)(n_boxes * box_rows) * 128u);
+                        const uint8_t* src = wbase + (size_t)kc * W_BYTES;
+                        bulk_g2s(ws, src, kTileBytes, full);
+                        if (PHASE == 0) bulk_g2s(ws + kTileBytes, src + kTileBytes, kTileBytes, full);
+                    }
                     for (int b = 0; b < n_boxes; ++b)
                         tma_2d(ws + W_BYTES + (uint32_t)(b * box_rows) * 128u, &act_map, kc * kTileK,
                                it.row_start + b * box_rows, full);
