@@ -264,8 +264,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                     __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.h) + row * a.f + (size_t)it.wb * kTileRows;
                     for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 16) {
                         float g[16], u[16];
-                        tc_ld16(t_row + (uint32_t)c0, g);
-                        tc_ld16(t_row + (uint32_t)(128 + c0), u);
+                        tc_ld16x2(t_row + (uint32_t)c0, t_row + (uint32_t)(128 + c0), g, u);
                         if (valid) {
                             uint32_t pk[8];
 #pragma unroll
@@ -283,13 +282,15 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 } else {
                     float* dst = a.y_packed + row * a.d + (size_t)it.wb * 256;
                     const int c_half = it.n_cols / 2;
-                    for (int c0 = half * c_half; c0 < half * c_half + c_half; c0 += 16) {
-                        float v[16];
-                        tc_ld16(t_row + (uint32_t)c0, v);
+                    for (int c0 = half * c_half; c0 < half * c_half + c_half; c0 += 32) {     // c_half is 64 or 128
+                        float v[16], v2[16];
+                        tc_ld16x2(t_row + (uint32_t)c0, t_row + (uint32_t)(c0 + 16), v, v2);
                         if (valid) {
                             float4* o = reinterpret_cast<float4*>(dst + c0);
 #pragma unroll
                             for (int n = 0; n < 4; ++n) o[n] = make_float4(v[4 * n], v[4 * n + 1], v[4 * n + 2], v[4 * n + 3]);
+#pragma unroll
+                            for (int n = 0; n < 4; ++n) o[4 + n] = make_float4(v2[4 * n], v2[4 * n + 1], v2[4 * n + 2], v2[4 * n + 3]);
                         }
                     }
                 }

@@ -331,6 +331,18 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
         const size_t out_ld = PHASE == 0 ? (size_t)a.f : (size_t)a.d;
         while (ok && walk.next(it)) {
             ok = mbar_wait(smem_u32(&bar_acc_full[acc]), acc_phase[acc], abort_p, a.status);
+            // The epilogue warps meet at named barriers below; if one of them gave up its wait, all of
+            // them must leave together (every warp reaches this vote because the wait is bounded).
+            {
+                uint32_t all_ok;
+                asm volatile(
+                    "{\n\t.reg .pred p, q;\n\t"
+                    "setp.ne.u32 q, %1, 0;\n\t"
+                    "bar.red.and.pred p, 1, 256, q;\n\t"
+                    "selp.u32 %0, 1, 0, p;\n\t}"
+                    : "=r"(all_ok) : "r"((uint32_t)ok) : "memory");
+                ok = all_ok != 0;
+            }
             if (!ok) break;
             tc_fence_after();
             const bool whole = it.kc_begin == 0 && it.kc_end == KC;
