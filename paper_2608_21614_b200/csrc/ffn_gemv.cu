@@ -14,8 +14,8 @@
 // pipes could not keep up with the weight stream.  Both operands take the SAME register-to-k
 // assignment (a lane's 16-byte chunk supplies k-slots {2t, 2t+1, 2t+8, 2t+9} of two MMAs), so the
 // contraction is exact without any shuffling of the loaded data.  The 8 warps of a CTA split the
-// k-chunks among themselves and their partial tiles are added in warp order through shared memory
-// (deterministic).
+// k-chunks (and, when the reduction length is short, several 16-row groups) among themselves and
+// their partial tiles are added in a fixed order through shared memory (deterministic).
 #include <cuda_bf16.h>
 
 #include "saem_internal.h"
@@ -38,7 +38,7 @@ __device__ __forceinline__ void mma_16816(float* c, const uint32_t a0, const uin
 // PHASE 0: h = silu(Wg x) * (Wu x);  PHASE 1: y = Wd h
 template <int PHASE>
 __global__ void __launch_bounds__(kGvThreads, 3)
-ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab) {
+ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, int gpc) {
     __shared__ int s_cnt[4];
     __shared__ int s_expert, s_row0, s_rows;
     __shared__ float red[kGvWarps][2][kGvRows][kGvMaxTokens];
@@ -83,7 +83,11 @@ ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab) {
 
     const int K = PHASE == 0 ? a.d : a.f;
     const int KC = K / kTileK;
-    const int rg = blockIdx.x;                 // 16-row group inside the expert's matrix
+    // A CTA owns gpc consecutive 16-row groups (more when the reduction length is short, so that every
+    // CTA still moves tens of KB); warp w works on group w % gpc and takes every (8 / gpc)-th k-chunk.
+    const int wpg = kGvWarps / gpc;            // warps per row group
+    const int rg = blockIdx.x * gpc + (warp % gpc);
+    const int kslice = warp / gpc;
     const int rb = rg >> 3, r_in = (rg & 7) * kGvRows;
     const int g = lane >> 2, t = lane & 3;     // MMA fragment coordinates
     const uint8_t* slot = a.slot_region + (size_t)tab.slot[e] * a.slot_bytes;
@@ -100,11 +104,11 @@ ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab) {
 
     float cg[4] = {0.f, 0.f, 0.f, 0.f}, cu[4] = {0.f, 0.f, 0.f, 0.f};
     constexpr int UN = PHASE == 0 ? 1 : 2;     // k-chunks of loads in flight per warp (three CTAs per SM)
-    for (int kc0 = warp; kc0 < KC; kc0 += kGvWarps * UN) {
+    for (int kc0 = kslice; kc0 < KC; kc0 += wpg * UN) {
         uint4 wl[UN][2], wh[UN][2], ul[UN][2], uh[UN][2], xv[UN][2];
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
-            const int kc = kc0 + u * kGvWarps;
+            const int kc = kc0 + u * wpg;
             if (kc < KC) {
                 const uint8_t* tile = wbase + (size_t)kc * chunk_stride;
                 wl[u][0] = *reinterpret_cast<const uint4*>(tile + off_lo0);
@@ -124,7 +128,7 @@ ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab) {
         }
 #pragma unroll
         for (int u = 0; u < UN; ++u) {
-            if (kc0 + u * kGvWarps < KC) {
+            if (kc0 + u * wpg < KC) {
 #pragma unroll
                 for (int b = 0; b < 2; ++b) {
                     mma_16816(cg, wl[u][b].x, wh[u][b].x, wl[u][b].y, wh[u][b].y, xv[u][b].x, xv[u][b].y);
@@ -149,17 +153,17 @@ ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab) {
         red[warp][1][g + 8][2 * t + 1] = cu[3];
     }
     __syncthreads();
-    if (tid < kGvRows * kGvMaxTokens) {
-        const int n = tid >> 4, r = tid & 15;      // 16 consecutive threads write 16 consecutive columns of one token row
+    // red[w] holds the partial tile of warp w = kslice * gpc + group; add a group's wpg slices in order
+    for (int o = tid; o < gpc * kGvRows * kGvMaxTokens; o += kGvThreads) {
+        const int grp = o >> 7, n = (o >> 4) & 7, r = o & 15;   // 16 consecutive threads: 16 consecutive columns of a token row
         if (n < m) {
             float sg = 0.f, su = 0.f;
-#pragma unroll
-            for (int w = 0; w < kGvWarps; ++w) {      // fixed warp order
-                sg += red[w][0][r][n];
-                if (PHASE == 0) su += red[w][1][r][n];
+            for (int ks = 0; ks < wpg; ++ks) {            // fixed order
+                sg += red[ks * gpc + grp][0][r][n];
+                if (PHASE == 0) su += red[ks * gpc + grp][1][r][n];
             }
             const size_t row = (size_t)(row0 + n);
-            const size_t col = (size_t)rg * kGvRows + r;
+            const size_t col = (size_t)(blockIdx.x * gpc + grp) * kGvRows + r;
             if (PHASE == 0) {
                 const float hv = sg / (1.f + expf(-sg)) * su;
                 reinterpret_cast<__nv_bfloat16*>(a.h)[row * a.f + col] = __float2bfloat16_rn(hv);
@@ -170,12 +174,23 @@ ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab) {
     }
 }
 
+// Row groups per CTA: enough that a CTA moves about 64 KB of weights, a power of two that divides
+// both the warp count and the number of row groups.
+static int groups_per_cta(int rows, int K, int matrices) {
+    const int n_groups = rows / kGvRows;
+    const long long bytes_per_group = (long long)kGvRows * K * 2 * matrices;
+    int gpc = 1;
+    while (gpc < kGvWarps && bytes_per_group * gpc < 64 * 1024 && n_groups % (gpc * 2) == 0) gpc *= 2;
+    return gpc;
+}
+
 cudaError_t launch_ffn_gemv(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch) {
     const int max_active = a.max_active < 1 ? 1 : a.max_active;
-    const dim3 g0((unsigned)(a.f / kGvRows), (unsigned)max_active), g1((unsigned)(a.d / kGvRows), (unsigned)max_active);
-    cudaError_t e = launch_pdl(ffn_gemv_kernel<0>, g0, dim3(kGvThreads), 0, st, a, tab);
+    const int gpc0 = groups_per_cta(a.f, a.d, 2), gpc1 = groups_per_cta(a.d, a.f, 1);
+    const dim3 g0((unsigned)(a.f / kGvRows / gpc0), (unsigned)max_active), g1((unsigned)(a.d / kGvRows / gpc1), (unsigned)max_active);
+    cudaError_t e = launch_pdl(ffn_gemv_kernel<0>, g0, dim3(kGvThreads), 0, st, a, tab, gpc0);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(ffn_gemv_kernel<1>, g1, dim3(kGvThreads), 0, st, a, tab);
+    e = launch_pdl(ffn_gemv_kernel<1>, g1, dim3(kGvThreads), 0, st, a, tab, gpc1);
     *n_launch = 2;
     return e;
 }
