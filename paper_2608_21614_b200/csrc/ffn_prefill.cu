@@ -10,8 +10,13 @@
 //     of two (512 columns) handed over tile by tile, so the epilogue of one tile overlaps the
 //     MMAs into the other.
 //   * gate and up land in the same accumulator tile (columns 0..127 and 128..255 of the same
-//     token lane), so SiLU(gate)*up is a per-thread operation and h is written once, bf16, with
-//     16-byte stores; y is written fp32 with 16-byte stores.
+//     token lane), so SiLU(gate)*up is a per-thread operation and h is written once, bf16.
+//   * An accumulator lane is a token row, so a thread's results are 64 contiguous bytes of ONE
+//     output row and a warp's direct stores would touch 32 different rows per instruction; that
+//     store traffic was measured to cost a third of the down projection's time (it also delays the
+//     copy warp's loads).  Each epilogue warp therefore stages its 32 rows x 64 bytes in shared
+//     memory (64-byte swizzle, conflict-free) and hands them to the TMA as one tile store; only the
+//     ragged last rows of a segment are stored directly, row by row.
 //   * One persistent CTA per SM; whole tiles are dealt round-robin in the order (expert, weight
 //     block, token tile), so the CTAs that run at the same time share a weight block and it is
 //     fetched from HBM once and re-read from L2.  No tile is split, nothing is reduced across CTAs.
@@ -29,7 +34,9 @@ constexpr int kPfThreads = 320;            // warp 0 copies, warp 1 MMA, warps 2
 constexpr int kPfStageW = 2 * kTileBytes;  // 256 weight rows x 64 k
 constexpr int kPfTileX = 128 * 128;        // one 128-token tile x 64 k
 constexpr int kPfMaxStages = 4;
-constexpr int kPfSmem = 4 * (kPfStageW + kPfTileX) + 1024;   // = 3 x (32 KB + 2 x 16 KB) + 1 KB as well
+constexpr int kPfStageArea = 4 * (kPfStageW + kPfTileX);     // = 3 x (32 KB + 2 x 16 KB) as well
+constexpr int kPfStoreBuf = 2048;          // per epilogue warp: 32 rows x 64 bytes on their way out
+constexpr int kPfSmem = kPfStageArea + 8 * kPfStoreBuf + 1024;
 constexpr int kPfPairHalfRounds = 3;       // two tiles per item only with at least this many such items per TWO CTAs
 
 struct PfPlan {
@@ -67,7 +74,8 @@ __device__ __forceinline__ void pf_decode(const PfPlan& plan, int it, int& curso
 // PHASE 0: h = silu(x Wg^T) * (x Wu^T);  PHASE 1: y = h Wd^T
 template <int PHASE>
 __global__ void __launch_bounds__(kPfThreads, 1)
-ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_constant__ CUtensorMap act_map) {
+ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_constant__ CUtensorMap act_map,
+                   const __grid_constant__ CUtensorMap out_map) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ PfPlan plan;
     __shared__ __align__(8) uint64_t bar_full[kPfMaxStages], bar_empty[kPfMaxStages], bar_acc_full[2], bar_acc_empty[2];
@@ -244,6 +252,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         const int q = warp & 3;                 // TMEM lane quarter = token rows 32q .. 32q+31
         const int half = (warp - 2) >> 2;       // which half of the tile's columns
         const int i = q * 32 + lane;            // token row inside the tile
+        const uint32_t store_buf = smem_base + (uint32_t)kPfStageArea + (uint32_t)(warp - 2) * kPfStoreBuf;
         int acc = 0, cursor = 0;
         uint32_t acc_phase[2] = {0u, 0u};
         bool ok = true;
@@ -258,39 +267,74 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ac * 256);
                 const int r = t * 128 + i;
                 const bool valid = r < it.rows_here;
+                const bool full_box = t * 128 + q * 32 + 32 <= it.rows_here;     // this warp's 32 rows all exist
+                const int box_row = it.row_start + t * 128 + q * 32;
                 const size_t row = (size_t)(it.row_start + r);
                 if (PHASE == 0) {
                     // h columns [64 half, 64 half + 64) of this f-block: gate at TMEM column c, up at 128 + c
                     __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.h) + row * a.f + (size_t)it.wb * kTileRows;
-                    for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 16) {
-                        float g[16], u[16];
-                        tc_ld16x2(t_row + (uint32_t)c0, t_row + (uint32_t)(128 + c0), g, u);
-                        if (valid) {
-                            uint32_t pk[8];
+                    for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            float g[16], u[16];
+                            tc_ld16x2(t_row + (uint32_t)(c0 + 16 * j), t_row + (uint32_t)(128 + c0 + 16 * j), g, u);
 #pragma unroll
                             for (int n = 0; n < 8; ++n) {
                                 const float h0 = __fdividef(g[2 * n], 1.f + __expf(-g[2 * n])) * u[2 * n];
                                 const float h1 = __fdividef(g[2 * n + 1], 1.f + __expf(-g[2 * n + 1])) * u[2 * n + 1];
                                 __nv_bfloat162 p2 = __floats2bfloat162_rn(h0, h1);
-                                pk[n] = *reinterpret_cast<uint32_t*>(&p2);
+                                pk[8 * j + n] = *reinterpret_cast<uint32_t*>(&p2);
                             }
+                        }
+                        if (full_box) {
+                            if (lane == 0) bulk_wait_read();
+                            __syncwarp();
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                st_shared_v4(store_buf + (uint32_t)lane * 64u + (uint32_t)((c ^ ((lane >> 1) & 3)) << 4),
+                                             pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                tma_store_2d(&out_map, it.wb * kTileRows + c0, box_row, store_buf);
+                                bulk_commit();
+                            }
+                        } else if (valid) {
                             uint4* o = reinterpret_cast<uint4*>(dst + c0);
-                            o[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                            o[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) o[c] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
                         }
                     }
                 } else {
                     float* dst = a.y_packed + row * a.d + (size_t)it.wb * 256;
                     const int c_half = it.n_cols / 2;
                     for (int c0 = half * c_half; c0 < half * c_half + c_half; c0 += 32) {     // c_half is 64 or 128
-                        float v[16], v2[16];
-                        tc_ld16x2(t_row + (uint32_t)c0, t_row + (uint32_t)(c0 + 16), v, v2);
-                        if (valid) {
+                        float v[2][16];
+                        tc_ld16x2(t_row + (uint32_t)c0, t_row + (uint32_t)(c0 + 16), v[0], v[1]);
+                        if (full_box) {
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh) {
+                                if (lane == 0) bulk_wait_read();
+                                __syncwarp();
+#pragma unroll
+                                for (int c = 0; c < 4; ++c)
+                                    st_shared_v4(store_buf + (uint32_t)lane * 64u + (uint32_t)((c ^ ((lane >> 1) & 3)) << 4),
+                                                 __float_as_uint(v[hh][4 * c]), __float_as_uint(v[hh][4 * c + 1]),
+                                                 __float_as_uint(v[hh][4 * c + 2]), __float_as_uint(v[hh][4 * c + 3]));
+                                fence_proxy_async_smem();
+                                __syncwarp();
+                                if (lane == 0) {
+                                    tma_store_2d(&out_map, it.wb * 256 + c0 + 16 * hh, box_row, store_buf);
+                                    bulk_commit();
+                                }
+                            }
+                        } else if (valid) {
                             float4* o = reinterpret_cast<float4*>(dst + c0);
 #pragma unroll
-                            for (int n = 0; n < 4; ++n) o[n] = make_float4(v[4 * n], v[4 * n + 1], v[4 * n + 2], v[4 * n + 3]);
+                            for (int n = 0; n < 4; ++n) o[n] = make_float4(v[0][4 * n], v[0][4 * n + 1], v[0][4 * n + 2], v[0][4 * n + 3]);
 #pragma unroll
-                            for (int n = 0; n < 4; ++n) o[4 + n] = make_float4(v2[4 * n], v2[4 * n + 1], v2[4 * n + 2], v2[4 * n + 3]);
+                            for (int n = 0; n < 4; ++n) o[4 + n] = make_float4(v[1][4 * n], v[1][4 * n + 1], v[1][4 * n + 2], v[1][4 * n + 3]);
                         }
                     }
                 }
@@ -301,6 +345,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             }
             if (it.n_mt == 1) acc ^= 1;
         }
+        if (lane == 0) bulk_wait_all();         // this warp's tile stores have landed
     }
 
     // ---- teardown ----
@@ -325,13 +370,14 @@ cudaError_t ffn_prefill_init() {
 }
 
 cudaError_t launch_ffn_prefill(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x, const CUtensorMap& map_h,
-                               cudaStream_t st, int* n_launch) {
+                               const CUtensorMap& map_h_store, const CUtensorMap& map_y_store, cudaStream_t st,
+                               int* n_launch) {
     cudaError_t e = ffn_prefill_init();
     if (e != cudaSuccess) return e;
     const dim3 grid((unsigned)a.n_sm), block(kPfThreads);
-    e = launch_pdl(ffn_prefill_kernel<0>, grid, block, (size_t)kPfSmem, st, a, tab, map_x);
+    e = launch_pdl(ffn_prefill_kernel<0>, grid, block, (size_t)kPfSmem, st, a, tab, map_x, map_h_store);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(ffn_prefill_kernel<1>, grid, block, (size_t)kPfSmem, st, a, tab, map_h);
+    e = launch_pdl(ffn_prefill_kernel<1>, grid, block, (size_t)kPfSmem, st, a, tab, map_h, map_y_store);
     *n_launch = 2;
     return e;
 }

@@ -531,6 +531,17 @@ static bool make_act_map(CUtensorMap* m, const void* base, int rows, int K, int 
     return r == CUDA_SUCCESS;
 }
 
+// Store map of the tiled kernels' epilogue: boxes of 32 rows x 64 bytes, 64-byte swizzle.
+static bool make_store_map(CUtensorMap* m, void* base, CUtensorMapDataType dt, int elem_bytes, int rows, int cols) {
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * elem_bytes};
+    cuuint32_t box[2] = {(cuuint32_t)(64 / elem_bytes), 32u};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(m, dt, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch) {
     {
         cudaError_t e = ffn_tensor_init();
@@ -542,7 +553,12 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
     if (!make_act_map(&map_x, a.x_packed, a.max_rows, a.d, box_rows)) return cudaErrorInvalidValue;
     if (!make_act_map(&map_h, a.h, a.max_rows, a.f, box_rows)) return cudaErrorInvalidValue;
     // Segments that can exceed 64 rows are a dense contraction: tile them for the tensor cores.
-    if (a.n_tile > 64) return launch_ffn_prefill(a, tab, map_x, map_h, st, n_launch);
+    if (a.n_tile > 64) {
+        alignas(64) CUtensorMap map_h_store, map_y_store;
+        if (!make_store_map(&map_h_store, a.h, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.max_rows, a.f)) return cudaErrorInvalidValue;
+        if (!make_store_map(&map_y_store, a.y_packed, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.max_rows, a.d)) return cudaErrorInvalidValue;
+        return launch_ffn_prefill(a, tab, map_x, map_h, map_h_store, map_y_store, st, n_launch);
+    }
     // Small token tiles (decode): two CTAs per SM, each with half the shared memory, so that one
     // CTA's prologue, epilogue and split-item reduction overlap the other's streaming.
     const bool two_per_sm = a.n_tile <= 64;

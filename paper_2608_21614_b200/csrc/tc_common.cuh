@@ -65,6 +65,21 @@ __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+// Tile store shared -> global through a tensor map (bulk async-group completion).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// the committing thread's stores have finished READING their shared-memory source
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... have completed altogether
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// orders this thread's ordinary shared-memory writes before later async-proxy (TMA) reads of them
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -117,9 +132,12 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n) {
 }
 
 
-// Large-segment (prefill) kernels, ffn_prefill.cu.  The activation maps have 32-row boxes.
+// Large-segment (prefill) kernels, ffn_prefill.cu.  The activation maps (loads) have 64 x 32 boxes with
+// the 128-byte swizzle; the store maps (h bf16, y fp32) have 64-byte-wide, 32-row boxes with the
+// 64-byte swizzle.
 cudaError_t launch_ffn_prefill(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x,
-                               const CUtensorMap& map_h, cudaStream_t st, int* n_launch);
+                               const CUtensorMap& map_h, const CUtensorMap& map_h_store,
+                               const CUtensorMap& map_y_store, cudaStream_t st, int* n_launch);
 
 }  // namespace saem
 
