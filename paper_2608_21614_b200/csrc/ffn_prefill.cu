@@ -265,83 +265,97 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ac * 256);
+                // This warp's slice of the tile goes to registers in one batch and the accumulator is
+                // handed back at once: the stores below overlap the MMAs of the next tile.
+                uint32_t v[128];
+                const int c_half = PHASE == 0 ? 64 : it.n_cols / 2;      // output columns of this warp: 64 or 128
+                if (PHASE == 0) {     // gate at TMEM columns [64 half, +64), up at 128 + the same
+                    tc_ld32_issue(t_row + (uint32_t)(half * 64), v);
+                    tc_ld32_issue(t_row + (uint32_t)(half * 64 + 32), v + 32);
+                    tc_ld32_issue(t_row + (uint32_t)(128 + half * 64), v + 64);
+                    tc_ld32_issue(t_row + (uint32_t)(128 + half * 64 + 32), v + 96);
+                } else {
+                    tc_ld32_issue(t_row + (uint32_t)(half * c_half), v);
+                    tc_ld32_issue(t_row + (uint32_t)(half * c_half + 32), v + 32);
+                    if (c_half == 128) {
+                        tc_ld32_issue(t_row + (uint32_t)(half * c_half + 64), v + 64);
+                        tc_ld32_issue(t_row + (uint32_t)(half * c_half + 96), v + 96);
+                    }
+                }
+                tc_wait_ld();
+#pragma unroll
+                for (int g16 = 0; g16 < 8; ++g16) tc_reg_fence16(v + 16 * g16);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[ac]));
+                acc_phase[ac] ^= 1u;
+
                 const int r = t * 128 + i;
                 const bool valid = r < it.rows_here;
                 const bool full_box = t * 128 + q * 32 + 32 <= it.rows_here;     // this warp's 32 rows all exist
                 const int box_row = it.row_start + t * 128 + q * 32;
                 const size_t row = (size_t)(it.row_start + r);
+                const uint32_t my_buf = store_buf + (uint32_t)lane * 64u;
+                const uint32_t sw = (uint32_t)((lane >> 1) & 3);
                 if (PHASE == 0) {
-                    // h columns [64 half, 64 half + 64) of this f-block: gate at TMEM column c, up at 128 + c
-                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.h) + row * a.f + (size_t)it.wb * kTileRows;
-                    for (int c0 = half * 64; c0 < half * 64 + 64; c0 += 32) {
+                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.h) + row * a.f + (size_t)it.wb * kTileRows + half * 64;
+#pragma unroll
+                    for (int bx = 0; bx < 2; ++bx) {          // two boxes of 32 h columns
                         uint32_t pk[16];
 #pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            float g[16], u[16];
-                            tc_ld16x2(t_row + (uint32_t)(c0 + 16 * j), t_row + (uint32_t)(128 + c0 + 16 * j), g, u);
-#pragma unroll
-                            for (int n = 0; n < 8; ++n) {
-                                const float h0 = __fdividef(g[2 * n], 1.f + __expf(-g[2 * n])) * u[2 * n];
-                                const float h1 = __fdividef(g[2 * n + 1], 1.f + __expf(-g[2 * n + 1])) * u[2 * n + 1];
-                                __nv_bfloat162 p2 = __floats2bfloat162_rn(h0, h1);
-                                pk[8 * j + n] = *reinterpret_cast<uint32_t*>(&p2);
-                            }
+                        for (int n = 0; n < 16; ++n) {
+                            const float g0 = __uint_as_float(v[32 * bx + 2 * n]), g1 = __uint_as_float(v[32 * bx + 2 * n + 1]);
+                            const float u0 = __uint_as_float(v[64 + 32 * bx + 2 * n]), u1 = __uint_as_float(v[64 + 32 * bx + 2 * n + 1]);
+                            const float h0 = __fdividef(g0, 1.f + __expf(-g0)) * u0;
+                            const float h1 = __fdividef(g1, 1.f + __expf(-g1)) * u1;
+                            __nv_bfloat162 p2 = __floats2bfloat162_rn(h0, h1);
+                            pk[n] = *reinterpret_cast<uint32_t*>(&p2);
                         }
                         if (full_box) {
                             if (lane == 0) bulk_wait_read();
                             __syncwarp();
 #pragma unroll
                             for (int c = 0; c < 4; ++c)
-                                st_shared_v4(store_buf + (uint32_t)lane * 64u + (uint32_t)((c ^ ((lane >> 1) & 3)) << 4),
-                                             pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                                st_shared_v4(my_buf + ((((uint32_t)c) ^ sw) << 4), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
                             fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) {
-                                tma_store_2d(&out_map, it.wb * kTileRows + c0, box_row, store_buf);
+                                tma_store_2d(&out_map, it.wb * kTileRows + half * 64 + 32 * bx, box_row, store_buf);
                                 bulk_commit();
                             }
                         } else if (valid) {
-                            uint4* o = reinterpret_cast<uint4*>(dst + c0);
+                            uint4* o = reinterpret_cast<uint4*>(dst + 32 * bx);
 #pragma unroll
                             for (int c = 0; c < 4; ++c) o[c] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
                         }
                     }
                 } else {
-                    float* dst = a.y_packed + row * a.d + (size_t)it.wb * 256;
-                    const int c_half = it.n_cols / 2;
-                    for (int c0 = half * c_half; c0 < half * c_half + c_half; c0 += 32) {     // c_half is 64 or 128
-                        float v[2][16];
-                        tc_ld16x2(t_row + (uint32_t)c0, t_row + (uint32_t)(c0 + 16), v[0], v[1]);
-                        if (full_box) {
+                    float* dst = a.y_packed + row * a.d + (size_t)it.wb * 256 + half * c_half;
 #pragma unroll
-                            for (int hh = 0; hh < 2; ++hh) {
+                    for (int bx = 0; bx < 8; ++bx) {          // boxes of 16 y columns
+                        if (bx * 16 < c_half) {
+                            if (full_box) {
                                 if (lane == 0) bulk_wait_read();
                                 __syncwarp();
 #pragma unroll
                                 for (int c = 0; c < 4; ++c)
-                                    st_shared_v4(store_buf + (uint32_t)lane * 64u + (uint32_t)((c ^ ((lane >> 1) & 3)) << 4),
-                                                 __float_as_uint(v[hh][4 * c]), __float_as_uint(v[hh][4 * c + 1]),
-                                                 __float_as_uint(v[hh][4 * c + 2]), __float_as_uint(v[hh][4 * c + 3]));
+                                    st_shared_v4(my_buf + ((((uint32_t)c) ^ sw) << 4), v[16 * bx + 4 * c], v[16 * bx + 4 * c + 1],
+                                                 v[16 * bx + 4 * c + 2], v[16 * bx + 4 * c + 3]);
                                 fence_proxy_async_smem();
                                 __syncwarp();
                                 if (lane == 0) {
-                                    tma_store_2d(&out_map, it.wb * 256 + c0 + 16 * hh, box_row, store_buf);
+                                    tma_store_2d(&out_map, it.wb * 256 + half * c_half + 16 * bx, box_row, store_buf);
                                     bulk_commit();
                                 }
+                            } else if (valid) {
+                                uint4* o = reinterpret_cast<uint4*>(dst + 16 * bx);
+#pragma unroll
+                                for (int c = 0; c < 4; ++c)
+                                    o[c] = make_uint4(v[16 * bx + 4 * c], v[16 * bx + 4 * c + 1], v[16 * bx + 4 * c + 2], v[16 * bx + 4 * c + 3]);
                             }
-                        } else if (valid) {
-                            float4* o = reinterpret_cast<float4*>(dst + c0);
-#pragma unroll
-                            for (int n = 0; n < 4; ++n) o[n] = make_float4(v[0][4 * n], v[0][4 * n + 1], v[0][4 * n + 2], v[0][4 * n + 3]);
-#pragma unroll
-                            for (int n = 0; n < 4; ++n) o[4 + n] = make_float4(v[1][4 * n], v[1][4 * n + 1], v[1][4 * n + 2], v[1][4 * n + 3]);
                         }
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[ac]));
-                acc_phase[ac] ^= 1u;
             }
             if (it.n_mt == 1) acc ^= 1;
         }
