@@ -56,7 +56,7 @@ typedef enum saem_status {
 enum { SAEM_MAX_EXPERTS = 128 };         /* routed experts per layer */
 enum { SAEM_TEMP = -2 };                 /* slot argument of saem_cache_load: take a temporary slot */
 enum { SAEM_OUT_F32 = 0, SAEM_OUT_BF16 = 1 };
-enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2 };
+enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TENSOR_PAIRS = 3 };
 
 /*
  * Shape of one context.  d_model and d_ff must be multiples of 128, at most 16384; 1 <= top_k <= n_experts <=
@@ -68,7 +68,11 @@ enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2 };
  * ffn_path: SAEM_FFN_AUTO picks per call -- matrix-vector kernels when no segment can exceed 8
  * rows, the tcgen05 weight-streaming kernels up to 64 rows, the tcgen05 tiled kernels beyond;
  * SAEM_FFN_TENSOR always uses the tcgen05 kernels; SAEM_FFN_SCALAR forces the plain scalar
- * kernels (kept for triage).
+ * kernels (kept for triage).  The tiled kernels exist in two forms: one CTA per tile, and CTA pairs
+ * (tcgen05 cta_group::2: 256 tokens x 512 weight rows per pair of SMs), which AUTO and TENSOR take
+ * for long reductions and many rows (d_model >= 4096, d_model % 256 == 0, at least 1536 packed
+ * rows in the call); SAEM_FFN_TENSOR_PAIRS is SAEM_FFN_TENSOR with the pair form whenever
+ * d_model % 256 == 0 (for tests and measurements).
  * n_shared (0..16, n_experts + n_shared <= SAEM_MAX_EXPERTS): always-on shared experts of the same
  * width d_ff that run INSIDE the layer's grouped launch.  They are experts n_experts ..
  * n_experts + n_shared - 1 of every layer for the cache calls (outside the routed cache-ratio

@@ -542,6 +542,18 @@ static bool make_store_map(CUtensorMap* m, void* base, CUtensorMapDataType dt, i
     return r == CUDA_SUCCESS;
 }
 
+// The slot region as rows of 128 bytes; a box of 128 rows is one packed 16 KB weight tile, copied as it is.
+static bool make_weight_map(CUtensorMap* m, const void* base, size_t bytes) {
+    cuuint64_t dims[2] = {128, (cuuint64_t)(bytes >> 7)};
+    cuuint64_t strides[1] = {128};
+    cuuint32_t box[2] = {128, 128};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch) {
     {
         cudaError_t e = ffn_tensor_init();
@@ -557,6 +569,14 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
         alignas(64) CUtensorMap map_h_store, map_y_store;
         if (!make_store_map(&map_h_store, a.h, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.max_rows, a.f)) return cudaErrorInvalidValue;
         if (!make_store_map(&map_y_store, a.y_packed, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.max_rows, a.d)) return cudaErrorInvalidValue;
+        // CTA pairs pay when the reductions are long (their items use every accumulator column, so
+        // an item boundary costs more) and there are rows for several rounds of 256 x 512 items
+        const bool pairs_fit = a.d % 256 == 0 && a.n_sm >= 2 && (a.slot_region_bytes >> 7) < (1ull << 31);
+        if (pairs_fit && (a.force_pairs || (a.d >= 4096 && a.max_rows >= 1536))) {
+            alignas(64) CUtensorMap map_w;
+            if (!make_weight_map(&map_w, a.slot_region, a.slot_region_bytes)) return cudaErrorInvalidValue;
+            return launch_ffn_pair(a, tab, map_x, map_h, map_w, map_h_store, map_y_store, st, n_launch);
+        }
         return launch_ffn_prefill(a, tab, map_x, map_h, map_h_store, map_y_store, st, n_launch);
     }
     // Small token tiles (decode): two CTAs per SM, each with half the shared memory, so that one

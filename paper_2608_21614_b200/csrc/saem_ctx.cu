@@ -24,7 +24,7 @@ int validate_config(const saem_config* c) {
     if (c->temp_slots < 0 || c->temp_slots > 4096) return SAEM_ERR_SHAPE;
     if ((long long)c->n_layers * c->slots_per_layer + c->temp_slots < 1) return SAEM_ERR_SHAPE;
     if (c->out_dtype != SAEM_OUT_F32 && c->out_dtype != SAEM_OUT_BF16) return SAEM_ERR_INVALID_ARG;
-    if (c->ffn_path < SAEM_FFN_AUTO || c->ffn_path > SAEM_FFN_TENSOR) return SAEM_ERR_INVALID_ARG;
+    if (c->ffn_path < SAEM_FFN_AUTO || c->ffn_path > SAEM_FFN_TENSOR_PAIRS) return SAEM_ERR_INVALID_ARG;
     // repack keeps a [pairs/32][E] table of 16-bit counters in shared memory
     long long chunks = ((long long)c->max_tokens * c->top_k + 31) / 32;
     if (chunks * c->n_experts * 2 > 160 * 1024) return SAEM_ERR_UNSUPPORTED;
@@ -321,6 +321,7 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     a.E = ES; a.d = g.d_model; a.f = g.d_ff;
     a.slot_region = c->slot_region;
     a.slot_bytes = c->slot_bytes;
+    a.slot_region_bytes = c->slot_bytes * (size_t)(c->n_fixed_slots + c->cfg.temp_slots);
     a.h = (uint16_t*)(c->ws + c->lay.h);
     a.y_packed = y_packed;
     a.status = (int*)(c->ws + c->lay.status);
@@ -335,6 +336,7 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
         a.max_active = bound < ES ? (int)bound : ES;
     }
     a.n_sm = c->n_sm;
+    a.force_pairs = g.ffn_path == SAEM_FFN_TENSOR_PAIRS;
     int nl = 0;
     const int seg_bound = max_rows < g.max_tokens ? max_rows : g.max_tokens;     // a token picks an expert once
     if (g.ffn_path == SAEM_FFN_SCALAR) {

@@ -57,6 +57,26 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+// The same for a kernel that runs as clusters of two CTAs (grid.x must be even).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl_pairs(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args... args) {
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 // Function attributes (large dynamic shared memory) are per device: returns true the first time it is
 // called for the current device with this flag array.
 inline bool first_call_on_device(bool (&done)[64]) {
@@ -90,6 +110,7 @@ struct FfnArgs {
     int E, d, f;
     const uint8_t* slot_region;
     size_t slot_bytes;
+    size_t slot_region_bytes;   // whole region (every slot)
     uint16_t* h;                // [max_rows, f] bf16 workspace
     float* y_packed;            // [max_rows, d]
     int* status;
@@ -99,6 +120,7 @@ struct FfnArgs {
     int n_tile;                 // token tile for this launch (multiple of 16, <= 256)
     int max_active;             // upper bound of experts with rows: min(E, T * top_k + n_shared)
     int n_sm;
+    int force_pairs;            // tiled kernels: CTA pairs whenever the shape allows
 };
 cudaError_t launch_ffn_scalar(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
 cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);

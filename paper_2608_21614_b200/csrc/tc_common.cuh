@@ -153,12 +153,93 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n) {
 }
 
 
+// ------------------------------------------------------------------ CTA pairs (cta_group::2)
+// Two CTAs of a cluster share one MMA: each supplies its 128 rows of A and its half of B from its own
+// shared memory, CTA 0 (the leader) issues, each keeps its 128 accumulator lanes in its own TMEM.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same variable in CTA `cta` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t cta) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait on a barrier of this CTA that the other CTA of the pair arrives on.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    unsigned long long t0 = 0;
+    for (uint32_t i = 0;; ++i) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((i & 1023u) == 1023u) {
+            if (*abort_flag) return false;
+            unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicExch(status, SAEM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+// Tile load by one CTA of a pair into its own shared memory; completion is signalled on a barrier
+// that may live in the other CTA of the pair (a shared::cluster address).  No multicast.
+__device__ __forceinline__ void tma_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t cluster_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued
+// so far have completed.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+// Instruction descriptor of the pair MMA: bf16 x bf16 -> fp32, K-major operands, M = 256 (128 per CTA), N = n.
+__device__ __forceinline__ uint32_t idesc_bf16_pair(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
 // Large-segment (prefill) kernels, ffn_prefill.cu.  The activation maps (loads) have 64 x 32 boxes with
 // the 128-byte swizzle; the store maps (h bf16, y fp32) have 64-byte-wide, 32-row boxes with the
 // 64-byte swizzle.
 cudaError_t launch_ffn_prefill(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x,
                                const CUtensorMap& map_h, const CUtensorMap& map_h_store,
                                const CUtensorMap& map_y_store, cudaStream_t st, int* n_launch);
+// The same with CTA pairs (ffn_pair.cu): 256 tokens x 512 weight rows per pair.  map_w views the slot
+// region as rows of 128 bytes (boxes of 128 rows = one packed 16 KB tile).  Needs d_model % 256 == 0.
+cudaError_t launch_ffn_pair(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x, const CUtensorMap& map_h,
+                            const CUtensorMap& map_w, const CUtensorMap& map_h_store, const CUtensorMap& map_y_store,
+                            cudaStream_t st, int* n_launch);
 
 }  // namespace saem
 

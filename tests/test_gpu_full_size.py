@@ -33,13 +33,21 @@ def test_fine_grained_decode_full(oracle, name, T, routing):
     layer.close()
 
 
-def test_c3_prefill_2048_sampled(oracle):
+PAIRS = 3       # SAEM_FFN_TENSOR_PAIRS: the CTA-pair form of the tiled kernels wherever the shape allows
+
+
+@pytest.mark.parametrize("name,tokens,path", [("c3", 2048, TENSOR), ("c3", 2048, PAIRS), ("c2", 1024, TENSOR)],
+                         ids=["c3-one-cta-tiles", "c3-cta-pairs", "c2-cta-pairs-by-rule"])
+def test_prefill_sampled(oracle, name, tokens, path):
+    """Prefill-sized batches through the tiled kernels.  c3 at 2048 tokens takes the one-CTA tiles by
+    default and the CTA pairs when forced; the Mixtral-shaped c2 at 1024 tokens (d_model 4096, 2048
+    packed rows) takes the CTA pairs by the default rule."""
     import gpu_util as g
-    cfg = gen.layer_config("c3", tokens=2048)
+    cfg = gen.layer_config(name, tokens=tokens)
     li = gen.layer_inputs(cfg)
     T, k, E, d = cfg.tokens, cfg.top_k, cfg.n_experts, cfg.d_model
     P = T * k
-    layer = g.make_layer(li, TENSOR)
+    layer = g.make_layer(li, path)
     out = layer.step(g.dev(li.logits), g.dev(li.x), T)
     torch.cuda.synchronize()
     assert layer.device_status() == 0
@@ -65,14 +73,16 @@ def test_c3_prefill_2048_sampled(oracle):
     y_gpu = g.host(layer.y_packed[:P])
     g.assert_close(y_gpu[rows], y_ref, "sampled y_packed rows")
     # shared expert: sampled tokens
-    toks = np.sort(rng.choice(T, 48, replace=False))
-    s_ref = oracle.expert_ffn(li.x[toks], np.array([0, len(toks)], np.int32), [li.shared[0]], [li.shared[1]],
-                              [li.shared[2]])
-    s_gpu = g.host(layer.shared_rows(T))
-    g.assert_close(s_gpu[toks], s_ref, "sampled shared rows")
+    s_gpu = None
+    if li.shared is not None:
+        toks = np.sort(rng.choice(T, 48, replace=False))
+        s_ref = oracle.expert_ffn(li.x[toks], np.array([0, len(toks)], np.int32), [li.shared[0]], [li.shared[1]],
+                                  [li.shared[2]])
+        s_gpu = g.host(layer.shared_rows(T))
+        g.assert_close(s_gpu[toks], s_ref, "sampled shared rows")
     # combine: in full, from the GPU's own FFN outputs (isolates the merge)
     c_ref = oracle.combine(y_gpu.astype(np.float64), ri, g.host(layer.topk_w).astype(np.float64),
-                           s_gpu.astype(np.float64))
+                           None if s_gpu is None else s_gpu.astype(np.float64))
     assert np.abs(g.host(out).astype(np.float64) - c_ref).max() <= 1e-4
     # properties that hold at any size: finite outputs, plausible scale
     o = g.host(out)

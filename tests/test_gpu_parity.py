@@ -9,7 +9,7 @@ from paper_2608_21614_b200 import inputs as gen
 
 pytestmark = pytest.mark.gpu
 
-AUTO, SCALAR, TENSOR = 0, 1, 2
+AUTO, SCALAR, TENSOR, PAIRS = 0, 1, 2, 3
 
 
 @pytest.fixture(scope="module")
@@ -54,6 +54,25 @@ def test_tiny_batches_matrix_vector_path(oracle, T, E, k, d, f, fs):
     layer.close()
 
 
+@pytest.mark.parametrize("T,E,k,d,f,fs", [
+    (300, 8, 2, 256, 256, 0),        # one pair of weight blocks in gate/up, a single block in down
+    (700, 12, 3, 512, 384, 384),     # odd number of f-blocks (a one-block item), in-layer shared expert, ragged tiles
+    (1500, 16, 2, 256, 640, 0),      # several 256-token tiles per expert, five f-blocks
+])
+def test_cta_pair_tiles(oracle, T, E, k, d, f, fs):
+    """The cta_group::2 form of the tiled kernels (forced: the default rule wants d_model >= 4096)."""
+    g = _g()
+    cfg = gen.LayerConfig("t", d, f, E, k, T, fs, "zipf", 1.1, seed=3 * T + E)
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, PAIRS)
+    g.run_stepwise_and_compare(layer, li, oracle)
+    y1, o1 = layer.y_packed.clone(), layer.out.clone()
+    layer.step(g.dev(li.logits), g.dev(li.x), li.cfg.tokens)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, layer.y_packed) and torch.equal(o1, layer.out)      # run to run: bit-identical
+    layer.close()
+
+
 @pytest.mark.parametrize("path", [SCALAR, TENSOR], ids=["scalar", "tensor"])
 @pytest.mark.parametrize("T,E,k,d,f,fs", [
     (1, 1, 1, 128, 128, 0),          # dense FFN, one token
@@ -73,7 +92,7 @@ def test_small_shapes(oracle, path, T, E, k, d, f, fs):
     layer.close()
 
 
-@pytest.mark.parametrize("path", [SCALAR, TENSOR], ids=["scalar", "tensor"])
+@pytest.mark.parametrize("path", [SCALAR, TENSOR, PAIRS], ids=["scalar", "tensor", "cta-pairs"])
 def test_segment_sizes_around_tile_edges(oracle, path):
     """One expert, k = 1: the segment is the whole batch; sizes straddle every tile boundary."""
     g = _g()
