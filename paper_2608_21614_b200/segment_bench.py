@@ -62,7 +62,9 @@ def main():
         us = a.elapsed_time(b) / args.steps * 1e3
         status = B.saem_last_device_status(ctx.handle)
         rows.append({"rows": n, "us": us, "weight_gbs": 3 * d * f * 2 / us / 1e3, "tflops": 6.0 * n * d * f / us / 1e6,
-                     "kernels": ("tiled tcgen05 (tokens as M)" if n > 64 else "streaming tcgen05 (weights as M)" if n > 8
+                     "kernels": ("tiled tcgen05 on CTA pairs (tokens as M)" if n >= 1536 and d >= 4096 and d % 256 == 0
+                                 else "tiled tcgen05 (tokens as M)" if n > 64
+                                 else "streaming tcgen05 (weights as M)" if n > 8
                                  else "matrix-vector (mma.sync)"), "status": status})
         ctx.close()
     print(json.dumps({"d_model": d, "d_ff": f, "copies": args.copies, "peaks": {k: peaks.get(k) for k in
