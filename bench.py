@@ -174,14 +174,23 @@ def run_ours(args):
     launches0 = layer.launches()
     # timed region 1: exactly K steps, nothing between the kernels of a step (an event recorded
     # between two launches would forbid their programmatic overlap) -> the headline value
-    ev0.record(stream)
-    for i in range(K):
-        layer.step(logits_all[i % n_draws], x, T)
-    ev1.record(stream)
+    if args.graph:      # the step of every routing draw recorded once; the timed loop replays them
+        graphs = [layer.capture_step(lg, x, T) for lg in logits_all]
+        per_step = (layer.launches() - launches0) // (2 * n_draws)      # capture_step runs the step twice
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for i in range(K):
+            graphs[i % n_draws].replay()
+        ev1.record(stream)
+    else:
+        ev0.record(stream)
+        for i in range(K):
+            layer.step(logits_all[i % n_draws], x, T)
+        ev1.record(stream)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    launches = layer.launches() - launches0
+    launches = per_step * K if args.graph else layer.launches() - launches0
     total_ms = ev0.elapsed_time(ev1)
     # timed region 2: the same K steps with CUDA events around the saem_expert_ffn call(s) -> the
     # dominant kernel's duration for the roofline
@@ -240,6 +249,7 @@ def run_ours(args):
                        "routing": "%s popularity + Gumbel, seed 0" % cfg.routing, "cache": "all experts resident in HBM",
                        "l2": "layer weights %.2f GB vs 126 MB L2: inputs larger than L2, no flush" % weight_gb,
                        "distinct_weight_sets": args.distinct, "replicas": world,
+                       "launch": "CUDA-graph replay of the step" if args.graph else "one host call per kernel group",
                        "timing": "value: K steps back to back; roofline: a second pass of K steps with events around the FFN call"},
             "roofline": roof,
             "e2e": {"value": world * T / e2e_step_s, "unit": UNIT, "h2d_bytes_per_step": T * E * 4 + T * d * 2,
@@ -321,6 +331,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--distinct", type=int, default=8, help="distinct expert weight sets to generate (1..8)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
+    ap.add_argument("--graph", action="store_true", help="time CUDA-graph replays of the step (for steps of a few tens of us)")
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS), help="c2 is the benchmark; c3/c4 for study")
     ap.add_argument("--tokens", type=int, default=None, help="override the batch of the workload")
     ap.add_argument("--routing", default=None, choices=["zipf", "uniform", "normal"])

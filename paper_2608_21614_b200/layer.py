@@ -120,6 +120,22 @@ class MoELayer:
         self.combine(T, stream)
         return self.out[:T]
 
+    def capture_step(self, logits: torch.Tensor, x: torch.Tensor, T: int, layer: int = 0) -> "torch.cuda.CUDAGraph":
+        """The same five launches recorded once as a CUDA graph (every call of the library only
+        enqueues on the stream it is given, so a step can be captured).  `replay()` re-runs the step
+        on the current contents of `logits` and `x`; at batch 1 a step is short enough that issuing
+        five launches from the host costs more than running them."""
+        side = torch.cuda.Stream(device=self.device)
+        side.wait_stream(torch.cuda.current_stream(self.device))
+        with torch.cuda.stream(side):
+            self.step(logits, x, T, layer)          # warm-up outside the capture (first-call set-up, tensor maps)
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                self.step(logits, x, T, layer)
+        torch.cuda.current_stream(self.device).wait_stream(side)
+        return graph
+
     def step_fused_call(self, logits: torch.Tensor, x: torch.Tensor, T: int, out: torch.Tensor, layer: int = 0,
                         stream=None):
         """The same step through the single saem_moe_step call (intermediates in the workspace)."""

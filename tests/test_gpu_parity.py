@@ -318,6 +318,30 @@ def test_step_is_graph_capturable_and_replays_identically(oracle):
     layer.close()
 
 
+def test_capture_step_helper_batch_1(oracle):
+    """MoELayer.capture_step at batch 1 (matrix-vector kernels): replays equal the eager step and follow new inputs."""
+    g = _g()
+    cfg = gen.LayerConfig("t", 256, 384, 60, 4, 1, 384, "zipf", 1.1, seed=11)
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, AUTO)
+    logits, x = g.dev(li.logits), g.dev(li.x)
+    eager = layer.step(logits, x, 1).clone()
+    graph = layer.capture_step(logits, x, 1)
+    layer.out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(layer.out[:1], eager)
+    li2 = gen.layer_inputs(dataclasses.replace(cfg, seed=12))
+    logits.copy_(g.dev(li2.logits))
+    x.copy_(g.dev(li2.x))
+    graph.replay()
+    torch.cuda.synchronize()
+    ref = oracle.moe_step(li2.logits, li2.x, cfg.top_k, li.gate, li.up, li.down, shared=li.shared)
+    g.assert_close(g.host(layer.out[:1]), ref["out"], "graph replay, batch 1, new inputs")
+    assert layer.device_status() == 0
+    layer.close()
+
+
 def test_empty_batch_and_limits(B):
     """T = 0 is a no-op everywhere (repack still zeroes counts and offsets); T = max_tokens works and
     T = max_tokens + 1 is refused before anything is enqueued."""
