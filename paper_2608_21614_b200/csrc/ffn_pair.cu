@@ -72,7 +72,7 @@ __device__ __forceinline__ void pr_decode(const PrPlan& plan, int it, int& curso
 template <int PHASE>
 __global__ void __launch_bounds__(kPrThreads, 1)
 ffn_pair_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_constant__ CUtensorMap act_map,
-                const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap out_map) {
+                const __grid_constant__ CUtensorMap act_map128, const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap out_map) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ PrPlan plan;
     __shared__ __align__(8) uint64_t bar_full[kPrStages], bar_empty[kPrStages], bar_acc_full[2], bar_acc_empty[2];
@@ -189,9 +189,13 @@ ffn_pair_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_c
                     if (rank == 0) mbar_expect_tx(smem_u32(&bar_full[stage]), bytes);
                     for (int j = 0; j < it.n_wb; ++j)
                         tma_2d_pair(ws + (uint32_t)j * kTileBytes, &w_map, 0, w_row[j] + kc * w_row_step, full);
-                    for (int b = 0; b < n_boxes; ++b)
-                        tma_2d_pair(ws + 2u * kTileBytes + (uint32_t)b * 4096u, &act_map, kc * kTileK,
-                                    it.row_start + 128 * (int)rank + b * 32, full);
+                    if (n_boxes == 4) {     // a whole 128-token tile in one copy
+                        tma_2d_pair(ws + 2u * kTileBytes, &act_map128, kc * kTileK, it.row_start + 128 * (int)rank, full);
+                    } else {
+                        for (int b = 0; b < n_boxes; ++b)
+                            tma_2d_pair(ws + 2u * kTileBytes + (uint32_t)b * 4096u, &act_map, kc * kTileK,
+                                        it.row_start + 128 * (int)rank + b * 32, full);
+                    }
                 }
                 ++issued;
                 if (++stage == kPrStages) { stage = 0; phase ^= 1u; }
@@ -365,7 +369,7 @@ ffn_pair_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_c
 static bool g_pr_init[64];
 
 cudaError_t launch_ffn_pair(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x, const CUtensorMap& map_h,
-                            const CUtensorMap& map_w, const CUtensorMap& map_h_store, const CUtensorMap& map_y_store,
+                            const CUtensorMap& map_x128, const CUtensorMap& map_h128, const CUtensorMap& map_w, const CUtensorMap& map_h_store, const CUtensorMap& map_y_store,
                             cudaStream_t st, int* n_launch) {
     if (first_call_on_device(g_pr_init)) {
         cudaError_t e = cudaFuncSetAttribute(ffn_pair_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrSmem);
@@ -374,9 +378,9 @@ cudaError_t launch_ffn_pair(const FfnArgs& a, const SlotTable& tab, const CUtens
         if (e != cudaSuccess) return e;
     }
     const dim3 grid((unsigned)(a.n_sm & ~1)), block(kPrThreads);
-    cudaError_t e = launch_pdl_pairs(ffn_pair_kernel<0>, grid, block, (size_t)kPrSmem, st, a, tab, map_x, map_w, map_h_store);
+    cudaError_t e = launch_pdl_pairs(ffn_pair_kernel<0>, grid, block, (size_t)kPrSmem, st, a, tab, map_x, map_x128, map_w, map_h_store);
     if (e != cudaSuccess) return e;
-    e = launch_pdl_pairs(ffn_pair_kernel<1>, grid, block, (size_t)kPrSmem, st, a, tab, map_h, map_w, map_y_store);
+    e = launch_pdl_pairs(ffn_pair_kernel<1>, grid, block, (size_t)kPrSmem, st, a, tab, map_h, map_h128, map_w, map_y_store);
     *n_launch = 2;
     return e;
 }

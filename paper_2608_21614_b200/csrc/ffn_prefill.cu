@@ -75,6 +75,7 @@ __device__ __forceinline__ void pf_decode(const PfPlan& plan, int it, int& curso
 template <int PHASE>
 __global__ void __launch_bounds__(kPfThreads, 1)
 ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid_constant__ CUtensorMap act_map,
+                   const __grid_constant__ CUtensorMap act_map128, const __grid_constant__ CUtensorMap act_map256,
                    const __grid_constant__ CUtensorMap out_map) {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ PfPlan plan;
@@ -188,9 +189,22 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                     const uint32_t full = smem_u32(&bar_full[stage]);
                     const uint32_t ws = smem_base + (uint32_t)stage * stage_bytes;
                     mbar_expect_tx(full, w_bytes + (uint32_t)n_boxes * 4096u);
-                    bulk_g2s(ws, w0 + (size_t)kc * w_step, kTileBytes, full);
-                    if (it.n_cols == 256) bulk_g2s(ws + kTileBytes, w1 + (size_t)kc * w_step, kTileBytes, full);
-                    for (int b = 0; b < n_boxes; ++b)
+                    // few, large copies: issuing them is serial work of this one thread on the refill path
+                    if (PHASE == 0) {       // the gate tile and the up tile of a chunk are adjacent
+                        bulk_g2s(ws, w0 + (size_t)kc * w_step, kPfStageW, full);
+                    } else {
+                        bulk_g2s(ws, w0 + (size_t)kc * w_step, kTileBytes, full);
+                        if (it.n_cols == 256) bulk_g2s(ws + kTileBytes, w1 + (size_t)kc * w_step, kTileBytes, full);
+                    }
+                    // whole token tiles in one copy (256 or 128 rows), the ragged rest in 32-row boxes
+                    int b = 0;
+                    if (n_boxes == 8) {
+                        tma_2d(ws + kPfStageW, &act_map256, kc * kTileK, it.row_start, full);
+                        b = 8;
+                    }
+                    for (; b + 4 <= n_boxes; b += 4)
+                        tma_2d(ws + kPfStageW + (uint32_t)b * 4096u, &act_map128, kc * kTileK, it.row_start + b * 32, full);
+                    for (; b < n_boxes; ++b)
                         tma_2d(ws + kPfStageW + (uint32_t)b * 4096u, &act_map, kc * kTileK, it.row_start + b * 32, full);
                 }
                 ++issued;
@@ -384,14 +398,15 @@ cudaError_t ffn_prefill_init() {
 }
 
 cudaError_t launch_ffn_prefill(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x, const CUtensorMap& map_h,
-                               const CUtensorMap& map_h_store, const CUtensorMap& map_y_store, cudaStream_t st,
+                               const CUtensorMap& map_x128, const CUtensorMap& map_h128, const CUtensorMap& map_x256,
+                               const CUtensorMap& map_h256, const CUtensorMap& map_h_store, const CUtensorMap& map_y_store, cudaStream_t st,
                                int* n_launch) {
     cudaError_t e = ffn_prefill_init();
     if (e != cudaSuccess) return e;
     const dim3 grid((unsigned)a.n_sm), block(kPfThreads);
-    e = launch_pdl(ffn_prefill_kernel<0>, grid, block, (size_t)kPfSmem, st, a, tab, map_x, map_h_store);
+    e = launch_pdl(ffn_prefill_kernel<0>, grid, block, (size_t)kPfSmem, st, a, tab, map_x, map_x128, map_x256, map_h_store);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(ffn_prefill_kernel<1>, grid, block, (size_t)kPfSmem, st, a, tab, map_h, map_y_store);
+    e = launch_pdl(ffn_prefill_kernel<1>, grid, block, (size_t)kPfSmem, st, a, tab, map_h, map_h128, map_h256, map_y_store);
     *n_launch = 2;
     return e;
 }

@@ -566,7 +566,11 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
     if (!make_act_map(&map_h, a.h, a.max_rows, a.f, box_rows)) return cudaErrorInvalidValue;
     // Segments that can exceed 64 rows are a dense contraction: tile them for the tensor cores.
     if (a.n_tile > 64) {
-        alignas(64) CUtensorMap map_h_store, map_y_store;
+        alignas(64) CUtensorMap map_h_store, map_y_store, map_x128, map_h128, map_x256, map_h256;
+        if (!make_act_map(&map_x256, a.x_packed, a.max_rows, a.d, 256)) return cudaErrorInvalidValue;
+        if (!make_act_map(&map_h256, a.h, a.max_rows, a.f, 256)) return cudaErrorInvalidValue;
+        if (!make_act_map(&map_x128, a.x_packed, a.max_rows, a.d, 128)) return cudaErrorInvalidValue;
+        if (!make_act_map(&map_h128, a.h, a.max_rows, a.f, 128)) return cudaErrorInvalidValue;
         if (!make_store_map(&map_h_store, a.h, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.max_rows, a.f)) return cudaErrorInvalidValue;
         if (!make_store_map(&map_y_store, a.y_packed, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.max_rows, a.d)) return cudaErrorInvalidValue;
         // CTA pairs pay when the reductions are long (their items use every accumulator column, so
@@ -575,9 +579,9 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
         if (pairs_fit && (a.force_pairs || (a.d >= 4096 && a.max_rows >= 1536))) {
             alignas(64) CUtensorMap map_w;
             if (!make_weight_map(&map_w, a.slot_region, a.slot_region_bytes)) return cudaErrorInvalidValue;
-            return launch_ffn_pair(a, tab, map_x, map_h, map_w, map_h_store, map_y_store, st, n_launch);
+            return launch_ffn_pair(a, tab, map_x, map_h, map_x128, map_h128, map_w, map_h_store, map_y_store, st, n_launch);
         }
-        return launch_ffn_prefill(a, tab, map_x, map_h, map_h_store, map_y_store, st, n_launch);
+        return launch_ffn_prefill(a, tab, map_x, map_h, map_x128, map_h128, map_x256, map_h256, map_h_store, map_y_store, st, n_launch);
     }
     // Small token tiles (decode): two CTAs per SM, each with half the shared memory, so that one
     // CTA's prologue, epilogue and split-item reduction overlap the other's streaming.

@@ -230,15 +230,16 @@ __device__ __forceinline__ uint32_t idesc_bf16_pair(int n) {
 }
 
 // Large-segment (prefill) kernels, ffn_prefill.cu.  The activation maps (loads) have 64 x 32 boxes with
-// the 128-byte swizzle; the store maps (h bf16, y fp32) have 64-byte-wide, 32-row boxes with the
+// the 128-byte swizzle (ragged tiles) and 64 x 128 / 64 x 256 boxes (whole token tiles in one copy); the store maps (h bf16, y fp32) have 64-byte-wide, 32-row boxes with the
 // 64-byte swizzle.
 cudaError_t launch_ffn_prefill(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x,
-                               const CUtensorMap& map_h, const CUtensorMap& map_h_store,
+                               const CUtensorMap& map_h, const CUtensorMap& map_x128, const CUtensorMap& map_h128,
+                               const CUtensorMap& map_x256, const CUtensorMap& map_h256, const CUtensorMap& map_h_store,
                                const CUtensorMap& map_y_store, cudaStream_t st, int* n_launch);
 // The same with CTA pairs (ffn_pair.cu): 256 tokens x 512 weight rows per pair.  map_w views the slot
 // region as rows of 128 bytes (boxes of 128 rows = one packed 16 KB tile).  Needs d_model % 256 == 0.
 cudaError_t launch_ffn_pair(const FfnArgs& a, const SlotTable& tab, const CUtensorMap& map_x, const CUtensorMap& map_h,
-                            const CUtensorMap& map_w, const CUtensorMap& map_h_store, const CUtensorMap& map_y_store,
+                            const CUtensorMap& map_x128, const CUtensorMap& map_h128, const CUtensorMap& map_w, const CUtensorMap& map_h_store, const CUtensorMap& map_y_store,
                             cudaStream_t st, int* n_launch);
 
 }  // namespace saem
