@@ -262,8 +262,7 @@ ffn_tensor_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __grid
                     if (!early_w) {
                         mbar_expect_tx(full, W_BYTES + (uint32_t)(n_boxes * box_rows) * 128u);
                         const uint8_t* src = wbase + (size_t)kc * W_BYTES;
-                        bulk_g2s(ws, src, kTileBytes, full);
-                        if (PHASE == 0) bulk_g2s(ws + kTileBytes, src + kTileBytes, kTileBytes, full);
+                        bulk_g2s(ws, src, W_BYTES, full);        // gate/up: the two tiles of a chunk are adjacent
                     }
                     for (int b = 0; b < n_boxes; ++b)
                         tma_2d(ws + W_BYTES + (uint32_t)(b * box_rows) * 128u, &act_map, kc * kTileK,
