@@ -18,34 +18,78 @@ namespace saem {
 constexpr int kRepackThreads = 512;
 constexpr int kFusedPairs = 2048;
 
+// Row length (in 16-bit entries) of the [expert][chunk] table: at least n_chunks, and an odd number of
+// 32-bit words, so that the lanes of a warp, which touch the same chunk of different experts, fall
+// into different shared-memory banks (with a row of 384 entries all 32 lanes hit one bank).
+__host__ __device__ __forceinline__ int table_stride(int n_chunks) {
+    int s = (n_chunks + 1) & ~1;
+    if (((s >> 1) & 1) == 0) s += 2;
+    return s;
+}
+
 struct RepackSmem {
     int counts[SAEM_MAX_EXPERTS];
     int offsets[SAEM_MAX_EXPERTS + 1];
     int bad;
+    int pad_[2];            // sizeof is a multiple of 16: the chunk table behind it is cleared with 16-byte stores
 };
+static_assert(sizeof(RepackSmem) % 16 == 0, "the chunk table must start 16-byte aligned");
 
 // Shared-memory carve: [RepackSmem][chunk table uint16 n_chunks*E][rank uint8 P_padded][perm int32 P (fused only)]
+// e8 (optional, P bytes): the expert ids staged in shared memory by one sweep of coalesced loads
+// that are all in flight together (255 = invalid); without it every warp pays a global-memory
+// round trip per 32-pair chunk, which is most of the index kernel's time at prefill sizes.
 __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int P, int E, int S, int T, RepackSmem& sm,
-                                            uint16_t* table, uint8_t* rank, int32_t* perm_s, bool write_global,
+                                            uint16_t* table, uint8_t* rank, uint8_t* e8, int32_t* perm_s, bool write_global,
                                             int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                                             int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
                                             int* __restrict__ status) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
-    const int n_chunks = (P + 31) >> 5;
-    // table[e * n_chunks + c]: pairs of chunk c routed to expert e (expert-major, so that the scan
+    const int n_chunks = (P + 31) >> 5, tstride = table_stride(n_chunks);
+    const int id_bits = E > 1 ? 32 - __clz(E - 1) : 0;
+    // table[e * tstride + c]: pairs of chunk c routed to expert e (expert-major, so that the scan
     // down the chunks of one expert reads consecutive shared-memory words)
-    for (int i = tid; i < n_chunks * E; i += blockDim.x) table[i] = 0;
+    {   // the table starts 16-byte aligned; clear it with wide stores (the tail may spill into the rank
+        // array behind it, which is written later)
+        uint4* t4 = reinterpret_cast<uint4*>(table);
+        const int n16 = (tstride * E * 2 + 15) >> 4;
+        for (int i = tid; i < n16; i += blockDim.x) t4[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
     if (tid == 0) sm.bad = 0;
+    if (e8) {
+        __syncthreads();                             // sm.bad is cleared before anyone may set it
+        for (int p0 = tid; p0 < P; p0 += 4 * blockDim.x) {
+            int v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { const int p = p0 + u * blockDim.x; v[u] = p < P ? idx[p] : 0; }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int p = p0 + u * blockDim.x;
+                if (p < P) {
+                    const bool okv = v[u] >= 0 && v[u] < E;
+                    if (!okv) sm.bad = 1;
+                    e8[p] = okv ? (uint8_t)v[u] : (uint8_t)255;
+                }
+            }
+        }
+    }
     __syncthreads();
     for (int c = warp; c < n_chunks; c += n_warps) {
         int p = c * 32 + lane;
-        int e = p < P ? idx[p] : -1;
-        if (p < P && (e < 0 || e >= E)) { e = -1; sm.bad = 1; }
-        unsigned grp = __match_any_sync(0xffffffffu, e);
+        int e = p >= P ? -1 : e8 ? (e8[p] == 255 ? -1 : (int)e8[p]) : idx[p];
+        if (!e8 && p < P && (e < 0 || e >= E)) { e = -1; sm.bad = 1; }
+        // lanes with the same expert id: one ballot per bit of the id (the index phase runs on one SM
+        // and is bound by its instruction issue, so only the bits that E needs); invalid pairs are
+        // masked out and never use their rank
+        unsigned grp = __ballot_sync(0xffffffffu, e >= 0);
+        for (int b = 0; b < id_bits; ++b) {
+            const unsigned bal = __ballot_sync(0xffffffffu, (e >> b) & 1);
+            grp &= ((e >> b) & 1) ? bal : ~bal;
+        }
         int r = __popc(grp & ((1u << lane) - 1u));
         if (e >= 0) {
             rank[p] = (uint8_t)r;
-            if (r == 0) table[e * n_chunks + c] = (uint16_t)__popc(grp);
+            if (r == 0) table[e * tstride + c] = (uint16_t)__popc(grp);
         }
     }
     __syncthreads();
@@ -54,14 +98,14 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
         int run = 0;
         for (int c0 = 0; c0 < n_chunks; c0 += 32) {
             const int c = c0 + lane;
-            const int v = c < n_chunks ? table[e * n_chunks + c] : 0;
+            const int v = c < n_chunks ? table[e * tstride + c] : 0;
             int inc = v;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const int n = __shfl_up_sync(0xffffffffu, inc, o);
                 if (lane >= o) inc += n;
             }
-            if (c < n_chunks) table[e * n_chunks + c] = (uint16_t)(run + inc - v);
+            if (c < n_chunks) table[e * tstride + c] = (uint16_t)(run + inc - v);
             run += __shfl_sync(0xffffffffu, inc, 31);
         }
         if (lane == 0) sm.counts[e] = run;
@@ -93,13 +137,16 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
         if (tid == 0 && sm.bad) atomicExch(status, SAEM_ERR_INVALID_ARG);
     }
     for (int p = tid; p < P; p += blockDim.x) {
-        int e = idx[p];
+        int e = e8 ? (e8[p] == 255 ? -1 : (int)e8[p]) : idx[p];
         if (e < 0 || e >= E) { if (write_global) inv_perm[p] = -1; continue; }
-        int r = sm.offsets[e] + table[e * n_chunks + (p >> 5)] + rank[p];
+        int r = sm.offsets[e] + table[e * tstride + (p >> 5)] + rank[p];
         if (perm_s) perm_s[r] = p;
-        if (write_global) { perm[r] = p; inv_perm[p] = r; }
+        else if (write_global) perm[r] = p;
+        if (write_global) inv_perm[p] = r;
     }
     __syncthreads();
+    if (perm_s && write_global)                      // the permutation leaves through shared memory: coalesced stores
+        for (int r = tid; r < sm.offsets[E]; r += blockDim.x) perm[r] = perm_s[r];
 }
 
 __device__ __forceinline__ void copy_row(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int d,
@@ -119,11 +166,11 @@ repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict_
     const int P = T * k, n_chunks = (P + 31) >> 5;
     RepackSmem& sm = *reinterpret_cast<RepackSmem*>(smem_raw);
     uint16_t* table = reinterpret_cast<uint16_t*>(smem_raw + sizeof(RepackSmem));
-    size_t off = sizeof(RepackSmem) + (((size_t)n_chunks * E * 2 + 15) & ~(size_t)15);
+    size_t off = sizeof(RepackSmem) + (((size_t)table_stride(n_chunks) * E * 2 + 15) & ~(size_t)15);
     int32_t* perm_s = reinterpret_cast<int32_t*>(smem_raw + off);
     uint8_t* rank = smem_raw + off + (size_t)n_chunks * 32 * 4;
     for (int i = threadIdx.x; i < n_chunks * 32; i += blockDim.x) perm_s[i] = -1;
-    index_phase(idx, P, E, S, T, sm, table, rank, perm_s, blockIdx.x == 0, counts, offsets, perm, inv_perm, status);
+    index_phase(idx, P, E, S, T, sm, table, rank, nullptr, perm_s, blockIdx.x == 0, counts, offsets, perm, inv_perm, status);
     const int total = sm.offsets[E];                 // rows actually packed (pairs with a valid expert)
     // each CTA copies rows r = blockIdx.x, blockIdx.x + gridDim.x, ...; 128 threads per row
     const int sub = threadIdx.x >> 7, nsub = blockDim.x >> 7;
@@ -136,17 +183,19 @@ repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict_
 }
 
 __global__ void __launch_bounds__(1024)
-repack_index_kernel(const int32_t* __restrict__ idx, int T, int E, int S, int k, int32_t* __restrict__ counts,
-                    int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
-                    int* __restrict__ status) {
+repack_index_kernel(const int32_t* __restrict__ idx, int T, int E, int S, int k, int stage_ids,
+                    int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ perm,
+                    int32_t* __restrict__ inv_perm, int* __restrict__ status) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     pdl_wait();
     pdl_launch_dependents();
     const int P = T * k, n_chunks = (P + 31) >> 5;
     RepackSmem& sm = *reinterpret_cast<RepackSmem*>(smem_raw);
     uint16_t* table = reinterpret_cast<uint16_t*>(smem_raw + sizeof(RepackSmem));
-    uint8_t* rank = smem_raw + sizeof(RepackSmem) + (((size_t)n_chunks * E * 2 + 15) & ~(size_t)15);
-    index_phase(idx, P, E, S, T, sm, table, rank, nullptr, true, counts, offsets, perm, inv_perm, status);
+    uint8_t* rank = smem_raw + sizeof(RepackSmem) + (((size_t)table_stride(n_chunks) * E * 2 + 15) & ~(size_t)15);
+    uint8_t* e8 = stage_ids ? rank + (size_t)n_chunks * 32 : nullptr;
+    int32_t* perm_s = stage_ids > 1 ? reinterpret_cast<int32_t*>(rank + (size_t)n_chunks * 64) : nullptr;
+    index_phase(idx, P, E, S, T, sm, table, rank, e8, perm_s, true, counts, offsets, perm, inv_perm, status);
 }
 
 __global__ void __launch_bounds__(256)
@@ -169,7 +218,7 @@ cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, i
                           int32_t* offsets, int32_t* perm, int32_t* inv_perm, uint16_t* x_packed, int* status,
                           int n_sm, cudaStream_t st, int* n_launch) {
     const int P = T * k, n_chunks = (P + 31) >> 5;
-    size_t base = sizeof(RepackSmem) + (((size_t)n_chunks * E * 2 + 15) & ~(size_t)15);
+    size_t base = sizeof(RepackSmem) + (((size_t)table_stride(n_chunks) * E * 2 + 15) & ~(size_t)15);
     static bool attr_done[64];
     if (first_call_on_device(attr_done)) {
         cudaError_t e = cudaFuncSetAttribute(repack_index_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -188,8 +237,11 @@ cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, i
                           counts, offsets, perm, inv_perm, x_packed, status);
     }
     size_t smem = base + (size_t)n_chunks * 32;
-    cudaError_t e = launch_pdl(repack_index_kernel, dim3(1), dim3(1024), smem, st, idx, T, E, S, k, counts, offsets, perm,
-                               inv_perm, status);
+    // when they fit too: the expert ids staged in shared memory (1), and the permutation as well (2)
+    const int stage_ids = smem + (size_t)n_chunks * 32 * 5 <= 200 * 1024 ? 2 : smem + (size_t)n_chunks * 32 <= 200 * 1024 ? 1 : 0;
+    if (stage_ids) smem += (size_t)n_chunks * 32 * (stage_ids == 2 ? 5 : 1);
+    cudaError_t e = launch_pdl(repack_index_kernel, dim3(1), dim3(1024), smem, st, idx, T, E, S, k, stage_ids, counts,
+                               offsets, perm, inv_perm, status);
     if (e != cudaSuccess) return e;
     *n_launch = 2;
     return launch_pdl(repack_gather_kernel, dim3(n_sm * 4), dim3(256), 0, st, x, perm, offsets, T, E, S, k, d, x_packed);

@@ -28,6 +28,8 @@ int validate_config(const saem_config* c) {
     // repack keeps a [pairs/32][E] table of 16-bit counters in shared memory
     long long chunks = ((long long)c->max_tokens * c->top_k + 31) / 32;
     if (chunks * c->n_experts * 2 > 160 * 1024) return SAEM_ERR_UNSUPPORTED;
+    // ... next to a rank byte per pair (rows of the table are padded by up to three entries)
+    if ((chunks + 3) * c->n_experts * 2 + chunks * 32 + 2048 > 200 * 1024) return SAEM_ERR_UNSUPPORTED;
     return SAEM_OK;
 }
 
