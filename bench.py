@@ -39,7 +39,7 @@ WORKLOADS = {
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the two FFN kernels of one step of workload c2
 # with all 8 experts active, from the ncu capture summarised in profiles/ffn_tensor_c2_decode.md
-NCU_FFN_TRAFFIC_BYTES = {"c2": 2845366000}
+NCU_FFN_TRAFFIC_BYTES = {"c2": 2844872000}
 
 
 def measured_peaks():
