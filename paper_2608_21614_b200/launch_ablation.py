@@ -12,6 +12,14 @@ repacked batch:
 Outputs of the two modes are compared: identical bits on the matrix-vector path (no k-split), and
 equal up to fp32 summation order on the streaming path, whose k-split points depend on how many
 experts share the launch.
+
+With --bookkeeping the whole step is also run the way the paper describes its starting point
+(Sec. III "bookkeeping": a mask per expert, a gather of that expert's tokens, the expert's dense
+execution, a scatter-add of the weighted result): per active expert one `nonzero` on the routing
+mask (a host synchronisation), one row gather, one FFN call on the gathered rows, one `index_add_`.
+The mask, gather and scatter-add are library (torch) operations here, as they are in the paper's
+PyTorch baseline; only the expert FFN runs in this library's kernels (a second context that holds
+every expert as a one-expert "layer").  It is a measurement harness, not a product path.
 """
 from __future__ import annotations
 
@@ -31,6 +39,7 @@ def main():
     ap.add_argument("--tokens", type=int, default=8)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--distinct", type=int, default=4)
+    ap.add_argument("--bookkeeping", action="store_true", help="also time the whole step with per-expert mask / gather / scatter-add")
     args = ap.parse_args()
     cfg = gen.layer_config(args.workload, tokens=args.tokens)
     li = gen.layer_inputs(cfg, n_distinct_experts=args.distinct)
@@ -71,8 +80,72 @@ def main():
            "grouped": {"us": t_group, "launches": l_group}, "per_expert": {"us": t_each, "launches": l_each},
            "speedup_of_grouping": t_each / t_group, "outputs_bit_identical": same, "max_abs_difference": max_diff,
            "device_status": layer.device_status()}
+    if args.bookkeeping:
+        out["bookkeeping"] = bookkeeping_step(cfg, li, layer, logits, x, args.steps)
     print(json.dumps(out))
     layer.close()
+
+
+def bookkeeping_step(cfg, li, layer, logits, x, steps):
+    """Whole step, grouped (route, repack, grouped FFN, combine) against per-expert bookkeeping."""
+    T, E, d, k = cfg.tokens, cfg.n_experts, cfg.d_model, cfg.top_k
+    n_sh = cfg.d_ff_shared // cfg.d_ff if cfg.d_ff_shared else 0
+    # every expert (and every d_ff-wide part of the shared expert) as layer l of a one-expert context
+    one = MoELayer(d, cfg.d_ff, 1, 1, T, 0, n_layers=E + n_sh, slots_per_layer=1)
+    for e in range(E):
+        one.load_expert(e, 0, 0, li.gate[e], li.up[e], li.down[e])
+    for s_ in range(n_sh):
+        rows = slice(s_ * cfg.d_ff, (s_ + 1) * cfg.d_ff)
+        one.load_expert(E + s_, 0, 0, li.shared[0][rows], li.shared[1][rows], np.ascontiguousarray(li.shared[2][:, rows]))
+    one.drop_host_copies()
+    from . import binding as B
+    xg = torch.empty((T, d), dtype=torch.uint16, device="cuda")
+    yg = torch.empty((T, d), dtype=torch.float32, device="cuda")
+    out_b = torch.zeros((T, d), dtype=torch.float32, device="cuda")
+    calls = [0]
+
+    def book():
+        layer.route(logits, T)
+        out_b.zero_()
+        idx, w = layer.topk_idx[:T].to(torch.int64), layer.topk_w[:T]
+        for e in range(E):
+            tok, slot = (idx == e).nonzero(as_tuple=True)           # mask -> indices: synchronises with the host
+            n = int(tok.numel())
+            if n == 0:
+                continue
+            xg.view(torch.int16)[:n] = x.view(torch.int16)[tok]      # gather (bit patterns)
+            B.saem_expert_ffn(one.ctx.handle, e, xg, None, n, None, yg)
+            out_b.index_add_(0, tok, yg[:n] * w[tok, slot].unsqueeze(1))    # scatter-add
+            calls[0] += 1
+        for s_ in range(n_sh):                                      # shared expert: every token, weight 1
+            B.saem_expert_ffn(one.ctx.handle, E + s_, x, None, T, None, yg)
+            out_b.add_(yg[:T])
+            calls[0] += 1
+
+    def grouped():
+        layer.step(logits, x, T)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / steps * 1e3
+
+    t_g = timed(grouped)
+    ref = layer.out[:T].clone()
+    calls[0] = 0
+    t_b = timed(book)
+    res = {"grouped_step_us": t_g, "bookkeeping_step_us": t_b, "ffn_calls_per_step": calls[0] / (steps + 3),
+           "speedup": t_b / t_g, "max_abs_difference": float((ref - out_b).abs().max()),
+           "device_status": one.device_status()}
+    one.close()
+    return res
 
 
 if __name__ == "__main__":
