@@ -71,6 +71,12 @@ def test_cta_pair_tiles(oracle, T, E, k, d, f, fs):
     torch.cuda.synchronize()
     assert torch.equal(y1, layer.y_packed) and torch.equal(o1, layer.out)      # run to run: bit-identical
     layer.close()
+    # the pair MMA adds the same products in the same order as the one-CTA tiles: identical bits
+    single = g.make_layer(li, TENSOR)
+    single.step(g.dev(li.logits), g.dev(li.x), li.cfg.tokens)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, single.y_packed) and torch.equal(o1, single.out)
+    single.close()
 
 
 @pytest.mark.parametrize("path", [SCALAR, TENSOR], ids=["scalar", "tensor"])
