@@ -27,6 +27,11 @@
  *     saem_last_device_status(); kernels never trap and never wait without a bound.
  *   - The four step calls never synchronise and never read device results on the host.
  *   - A context is not thread-safe: calls on one context must come from one thread at a time.
+ *   - Calls on one context must also be ordered on the GPU (one stream, or events between streams):
+ *     the hidden activations, the partial tiles and arrival counters of split reductions and the
+ *     buffers of saem_moe_step live in the context's workspace, so two saem_expert_ffn or
+ *     saem_moe_step calls of one context whose kernels overlap corrupt each other.  Use one context
+ *     per concurrent stream.
  */
 #ifndef SAEM_H_
 #define SAEM_H_
@@ -160,7 +165,9 @@ int saem_route_fused(saem_ctx* ctx, const void* x, const void* w_router, int T, 
  * (pair stored at packed row r), inv_perm[T*top_k] (packed row of pair p), x_packed[T*top_k,
  * d_model] bf16 = x[perm[r] / top_k].  Segments are in ascending expert id and keep ascending pair
  * id inside (a stable counting sort), so the permutation is unique.  An index outside
- * [0, n_experts) sets the device status word and the pair is dropped from every output.
+ * [0, n_experts) sets the device status word (INVALID_ARG) and the pair is dropped from every output:
+ * its inv_perm entry is -1, the segments hold the valid pairs only, and the perm entries behind the
+ * last segment are -1.
  * With config.n_shared = S > 0 the outputs grow: counts[n_experts + S], offsets[n_experts + S + 1],
  * x_packed[T*(top_k + S), d_model]; shared expert s owns rows [T*top_k + s*T, T*top_k + (s+1)*T),
  * a copy of x, and offsets[n_experts] is T*top_k.
@@ -217,7 +224,8 @@ int saem_moe_step_host(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const flo
 
 /* Device pointers of the intermediates of the last saem_moe_step (inside the workspace), for
  * inspection by tests: 0 topk_idx, 1 topk_w, 2 counts, 3 offsets, 4 perm, 5 inv_perm, 6 x_packed,
- * 7 y_packed, 8 shared_y, 9 h (hidden activations).  NULL for an unknown id. */
+ * 7 y_packed, 8 shared_y, 9 h (hidden activations), 10 the 640 int32 arrival counters of items whose
+ * reduction is split across CTAs (zero between calls).  NULL for an unknown id. */
 void* saem_step_buffer(saem_ctx* ctx, int which);
 
 /*
@@ -269,7 +277,10 @@ enum { SAEM_STATIC_SCRATCH_ELEMS = 1 << 20 };
 int saem_expert_ffn_static(const void* x_packed, const int32_t* offsets, int n_experts, int max_rows,
                            int d_model, int d_ff, const void* packed_experts, float* y_packed, void* stream);
 
-/* Reads and clears the sticky device status word (synchronises the device). */
+/* Reads and clears the sticky device status word (synchronises the device).  When the word is
+ * SAEM_ERR_TIMEOUT the arrival counters of split reductions are cleared as well (a CTA that gave up
+ * its wait did not arrive), so that the context can be used again; the outputs of the call that
+ * timed out are undefined. */
 int saem_last_device_status(saem_ctx* ctx, int* code);
 
 /* Number of kernels this library has launched through `ctx` since creation (host counter). */

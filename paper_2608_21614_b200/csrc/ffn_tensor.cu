@@ -559,6 +559,7 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
         if (e != cudaSuccess) return e;
     }
     const int box_rows = a.n_tile >= 32 ? 32 : 16;
+    if (a.n_tile % box_rows) return cudaErrorInvalidValue;     // an activation stage is a whole number of boxes
     const int nt0 = a.n_tile < kGateUpMaxTile ? a.n_tile : kGateUpMaxTile, nt1 = a.n_tile;
     alignas(64) CUtensorMap map_x, map_h;
     if (!make_act_map(&map_x, a.x_packed, a.max_rows, a.d, box_rows)) return cudaErrorInvalidValue;

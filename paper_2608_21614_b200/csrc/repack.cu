@@ -3,8 +3,8 @@
 // that keeps ascending pair id inside a segment, so the permutation is unique and no atomics
 // decide an order.  The row gather moves 16 bytes per thread per access.
 //
-// Index phase, one CTA: warps take consecutive 32-pair chunks; within a chunk __match_any_sync
-// groups equal expert ids and a lane's rank is the number of lower lanes in its group; an
+// Index phase, one CTA: warps take consecutive 32-pair chunks; within a chunk one ballot per bit of
+// the expert id groups equal ids and a lane's rank is the number of lower lanes in its group; an
 // [expert][chunk] table of 16-bit counts is scanned down the chunks by one warp per expert;
 // a scan over the expert totals gives the segment offsets.
 //
@@ -147,6 +147,9 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
     __syncthreads();
     if (perm_s && write_global)                      // the permutation leaves through shared memory: coalesced stores
         for (int r = tid; r < sm.offsets[E]; r += blockDim.x) perm[r] = perm_s[r];
+    // pairs with an invalid expert id were dropped: the rows behind the last segment hold no pair
+    if (write_global)
+        for (int r = sm.offsets[E] + tid; r < P; r += blockDim.x) perm[r] = -1;
 }
 
 __device__ __forceinline__ void copy_row(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int d,
@@ -204,10 +207,12 @@ repack_gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__
                      uint16_t* __restrict__ x_packed) {
     pdl_wait();
     pdl_launch_dependents();
+    // with shared experts offsets[E] is T*k whatever was dropped; rows without a pair have perm -1
     const int total = S > 0 ? T * k : offsets[E];
     const int sub = threadIdx.x >> 6, nsub = blockDim.x >> 6;     // 64 threads per row
     for (int r = blockIdx.x * nsub + sub; r < total; r += gridDim.x * nsub) {
         int p = perm[r];
+        if (p < 0) continue;
         copy_row(x + (size_t)(p / k) * d, x_packed + (size_t)r * d, d, threadIdx.x & 63, 64);
     }
     for (int r = blockIdx.x * nsub + sub; r < S * T; r += gridDim.x * nsub)      // shared segments: x itself

@@ -39,7 +39,9 @@ WorkspaceLayout workspace_layout(const saem_config& c) {
     size_t P = (size_t)c.max_tokens * c.top_k, T = c.max_tokens, d = c.d_model, f = c.d_ff;
     size_t E = (size_t)c.n_experts + c.n_shared;            // experts with a segment: routed, then shared
     size_t R = P + (size_t)c.n_shared * T;                  // packed rows: pairs, then T rows per shared expert
+    // token tiles above 32 rows are loaded as 32-row boxes: keep them a whole number of boxes
     int nt = round_up(c.max_tokens < kMaxNTile ? c.max_tokens : kMaxNTile, 16);
+    if (nt > 32) nt = round_up(nt, 32);
     L.n_tile_max = nt;
     L.partial_slot_floats = (size_t)2 * nt * kTileRows;
     size_t off = 0;
@@ -232,12 +234,13 @@ int saem_pack_expert_host(const saem_config* cfg, const void* gate, const void* 
 }
 
 // ------------------------------------------------------------------------------------------- steps
+static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
 static int check_T(saem_ctx* c, int T) {
     if (!c) return SAEM_ERR_INVALID_ARG;
     if (T < 0 || T > c->cfg.max_tokens) return SAEM_ERR_SHAPE;
     return SAEM_OK;
 }
-static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
 
 int saem_route(saem_ctx* c, const float* logits, int T, int32_t* idx, float* w, void* stream) {
     int s = check_T(c, T);
@@ -277,21 +280,10 @@ int saem_repack(saem_ctx* c, const int32_t* idx, const void* x, int T, int32_t* 
     return SAEM_OK;
 }
 
-int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t* offsets, int max_rows,
-                    const int32_t* subset, int n_subset, float* y_packed, void* stream) {
-    if (!c) return SAEM_ERR_INVALID_ARG;
-    const saem_config& g = c->cfg;
-    if (layer < 0 || layer >= g.n_layers) return SAEM_ERR_INVALID_ARG;
-    if (max_rows < 0 || max_rows > g.max_tokens * (g.top_k + g.n_shared)) return SAEM_ERR_SHAPE;
-    if (max_rows == 0) return SAEM_OK;
-    if (!x_packed || !y_packed) return SAEM_ERR_INVALID_ARG;
+// Slot of every expert of `layer` for one FFN launch (fixed slot, else temporary binding, else -1),
+// and `st` ordered after the loads still in flight for those slots.
+static int resolve_slots(saem_ctx* c, int layer, const int32_t* subset, int n_subset, cudaStream_t st, SlotTable& tab) {
     const int ES = c->n_total;
-    if (!offsets && ES != 1) return SAEM_ERR_INVALID_ARG;
-    if (misaligned(x_packed) || misaligned(y_packed)) return SAEM_ERR_ALIGNMENT;
-    if (subset && n_subset < 0) return SAEM_ERR_INVALID_ARG;
-    cudaStream_t st = (cudaStream_t)stream;
-
-    SlotTable tab;
     const int32_t* so = c->slot_of + (size_t)layer * ES;
     const int32_t* to = c->temp_of + (size_t)layer * ES;
     for (int e = 0; e < SAEM_MAX_EXPERTS; ++e) { tab.slot[e] = -1; tab.in_subset[e] = 0; }
@@ -314,6 +306,44 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
         if (q == cudaSuccess) { c->ev_pending[s] = 0; continue; }
         if (q != cudaErrorNotReady) return SAEM_ERR_CUDA;
         CUDA_TRY(cudaStreamWaitEvent(st, c->ready_ev[s], 0));
+    }
+    return SAEM_OK;
+}
+
+// Book-keeping after an FFN of `layer` has been enqueued on `st`: later loads into the slots it reads
+// must wait for it.
+static int note_ffn_enqueued(saem_ctx* c, int layer, cudaStream_t st, const SlotTable& tab) {
+    c->last_stream[layer] = st;
+    c->ffn_seen[layer] = 1;
+    if (c->dynamic_residency) {
+        CUDA_TRY(cudaEventRecord(c->read_ev[layer], st));
+        c->read_recorded[layer] = 1;
+        for (int e = 0; e < c->n_total; ++e) {
+            int s = tab.slot[e];
+            if (s >= c->n_fixed_slots) c->temp_last_layer[s - c->n_fixed_slots] = layer;
+        }
+    }
+    return SAEM_OK;
+}
+
+int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t* offsets, int max_rows,
+                    const int32_t* subset, int n_subset, float* y_packed, void* stream) {
+    if (!c) return SAEM_ERR_INVALID_ARG;
+    const saem_config& g = c->cfg;
+    if (layer < 0 || layer >= g.n_layers) return SAEM_ERR_INVALID_ARG;
+    if (max_rows < 0 || max_rows > g.max_tokens * (g.top_k + g.n_shared)) return SAEM_ERR_SHAPE;
+    if (max_rows == 0) return SAEM_OK;
+    if (!x_packed || !y_packed) return SAEM_ERR_INVALID_ARG;
+    const int ES = c->n_total;
+    if (!offsets && ES != 1) return SAEM_ERR_INVALID_ARG;
+    if (misaligned(x_packed) || misaligned(y_packed)) return SAEM_ERR_ALIGNMENT;
+    if (subset && n_subset < 0) return SAEM_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    SlotTable tab;
+    {
+        int r = resolve_slots(c, layer, subset, n_subset, st, tab);
+        if (r != SAEM_OK) return r;
     }
 
     FfnArgs a;
@@ -349,17 +379,7 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
         CUDA_TRY(launch_ffn_tensor(a, tab, st, &nl));
     }
     c->launches += nl;
-    c->last_stream[layer] = st;
-    c->ffn_seen[layer] = 1;
-    if (c->dynamic_residency) {
-        CUDA_TRY(cudaEventRecord(c->read_ev[layer], st));
-        c->read_recorded[layer] = 1;
-        for (int e = 0; e < ES; ++e) {
-            int s = tab.slot[e];
-            if (s >= c->n_fixed_slots) c->temp_last_layer[s - c->n_fixed_slots] = layer;
-        }
-    }
-    return SAEM_OK;
+    return note_ffn_enqueued(c, layer, st, tab);
 }
 
 int saem_combine(saem_ctx* c, const float* y, const int32_t* inv_perm, const float* w, int T, const float* shared_y,
@@ -378,9 +398,9 @@ int saem_combine(saem_ctx* c, const float* y, const int32_t* inv_perm, const flo
 void* saem_step_buffer(saem_ctx* c, int which) {
     if (!c) return nullptr;
     const WorkspaceLayout& L = c->lay;
-    size_t offs[10] = {L.topk_idx, L.topk_w, L.counts, L.offsets, L.perm, L.inv_perm, L.x_packed, L.y_packed,
-                       L.shared_y, L.h};
-    if (which < 0 || which >= 10) return nullptr;
+    size_t offs[11] = {L.topk_idx, L.topk_w, L.counts, L.offsets, L.perm, L.inv_perm, L.x_packed, L.y_packed,
+                       L.shared_y, L.h, L.counters};
+    if (which < 0 || which >= 11) return nullptr;
     return c->ws + offs[which];
 }
 
@@ -402,6 +422,28 @@ int saem_moe_step(saem_ctx* c, saem_ctx* sh, int layer, const float* logits, con
     int32_t* inv = (int32_t*)(w + L.inv_perm);
     float* y = (float*)(w + L.y_packed);
     float* shy = (float*)(w + L.shared_y);
+    if (!sh && g.ffn_path == SAEM_FFN_AUTO && decode_fused_supported(T, g.top_k)) {
+        // The smallest decode batches: two launches for the whole step (gate + repack indices + gate/up,
+        // then down + merge); x_packed and y_packed are not produced.
+        if (layer < 0 || layer >= g.n_layers) return SAEM_ERR_INVALID_ARG;
+        if (misaligned(x) || misaligned(out)) return SAEM_ERR_ALIGNMENT;
+        cudaStream_t st = (cudaStream_t)stream;
+        SlotTable tab;
+        if ((s = resolve_slots(c, layer, nullptr, 0, st, tab)) != SAEM_OK) return s;
+        DecodeArgs a;
+        a.logits = logits; a.x = (const uint16_t*)x;
+        a.T = T; a.E = g.n_experts; a.S = g.n_shared; a.k = g.top_k; a.d = g.d_model; a.f = g.d_ff; a.renorm = g.renorm;
+        a.slot_region = c->slot_region; a.slot_bytes = c->slot_bytes;
+        a.h = (uint16_t*)(w + L.h);
+        a.out = out; a.out_bf16 = g.out_dtype == SAEM_OUT_BF16;
+        a.topk_idx = idx; a.topk_w = tw; a.counts = (int32_t*)(w + L.counts); a.offsets = offsets;
+        a.perm = (int32_t*)(w + L.perm); a.inv_perm = inv;
+        a.status = (int*)(w + L.status);
+        int nl = 0;
+        CUDA_TRY(launch_decode_fused(a, tab, c->n_sm, st, &nl));
+        c->launches += nl;
+        return note_ffn_enqueued(c, layer, st, tab);
+    }
     if ((s = saem_route(c, logits, T, idx, tw, stream)) != SAEM_OK) return s;
     if ((s = saem_repack(c, idx, x, T, (int32_t*)(w + L.counts), offsets, (int32_t*)(w + L.perm), inv,
                          w + L.x_packed, stream)) != SAEM_OK) return s;
@@ -445,27 +487,23 @@ int saem_cache_load(saem_ctx* c, int layer, int expert, int slot, const void* pi
     const saem_config& g = c->cfg;
     size_t le = (size_t)layer * c->n_total + expert;
     cudaStream_t cs = (cudaStream_t)copy_stream;
-    int gslot;
+    // Work out the slot first, enqueue the wait / copy / event, and only then change the host tables:
+    // if a CUDA call fails nothing is marked resident that was never copied.
+    int gslot, temp_index = -1;
     int wait_layer = -1;
     if (slot == SAEM_TEMP) {
         if (g.temp_slots < 1) return SAEM_ERR_INVALID_ARG;
         if (c->slot_of[le] >= 0) return SAEM_ERR_INVALID_ARG;
-        int t = c->next_temp;
-        c->next_temp = (t + 1) % g.temp_slots;
-        gslot = c->n_fixed_slots + t;
-        if (c->slot_owner[gslot] >= 0) c->temp_of[c->slot_owner[gslot]] = -1;   // drop the old binding
-        if (c->temp_of[le] >= 0) c->slot_owner[c->temp_of[le]] = -1;             // expert re-bound: free its old temp slot
-        wait_layer = c->temp_last_layer[t];
-        c->temp_of[le] = gslot;
+        temp_index = c->next_temp;
+        gslot = c->n_fixed_slots + temp_index;
+        wait_layer = c->temp_last_layer[temp_index];
     } else {
         if (slot < 0 || slot >= g.slots_per_layer) return SAEM_ERR_INVALID_ARG;
         if (c->slot_of[le] >= 0) return SAEM_ERR_INVALID_ARG;
         gslot = layer * g.slots_per_layer + slot;
         if (c->slot_owner[gslot] >= 0) return SAEM_ERR_SLOT_BUSY;
         wait_layer = layer;
-        c->slot_of[le] = gslot;
     }
-    c->slot_owner[gslot] = (int32_t)le;
     // the copy must not overtake an enqueued FFN that still reads the slot's previous content
     if (wait_layer >= 0 && !c->read_recorded[wait_layer] && c->ffn_seen[wait_layer]) {
         // fully resident configurations record no event per FFN: mark the tail of that layer's
@@ -478,7 +516,20 @@ int saem_cache_load(saem_ctx* c, int layer, int expert, int slot, const void* pi
     if (cudaMemcpyAsync(c->slot_region + (size_t)gslot * c->slot_bytes, pinned, c->slot_bytes, cudaMemcpyHostToDevice,
                         cs) != cudaSuccess)
         return SAEM_ERR_CUDA;
-    if (cudaEventRecord(c->ready_ev[gslot], cs) != cudaSuccess) return SAEM_ERR_CUDA;
+    if (cudaEventRecord(c->ready_ev[gslot], cs) != cudaSuccess) {
+        // the copy is enqueued but cannot be waited for: whatever the slot held is no longer valid
+        if (c->slot_owner[gslot] >= 0) { c->temp_of[c->slot_owner[gslot]] = -1; c->slot_owner[gslot] = -1; }
+        return SAEM_ERR_CUDA;
+    }
+    if (slot == SAEM_TEMP) {
+        c->next_temp = (temp_index + 1) % g.temp_slots;
+        if (c->slot_owner[gslot] >= 0) c->temp_of[c->slot_owner[gslot]] = -1;   // drop the old binding
+        if (c->temp_of[le] >= 0) c->slot_owner[c->temp_of[le]] = -1;             // expert re-bound: free its old temp slot
+        c->temp_of[le] = gslot;
+    } else {
+        c->slot_of[le] = gslot;
+    }
+    c->slot_owner[gslot] = (int32_t)le;
     c->ev_pending[gslot] = 1;
     c->ev_recorded[gslot] = 1;
     return SAEM_OK;
@@ -534,6 +585,9 @@ int saem_last_device_status(saem_ctx* c, int* code) {
     CUDA_TRY(cudaMemcpy(c->pinned_status, c->ws + c->lay.status, sizeof(int), cudaMemcpyDeviceToHost));
     *code = *c->pinned_status;
     CUDA_TRY(cudaMemset(c->ws + c->lay.status, 0, sizeof(int)));
+    // a CTA that gave up a bounded wait skipped its arrival on a split item's counter: start the next
+    // launch from clean counters (nothing is in flight after the synchronisation above)
+    if (*code == SAEM_ERR_TIMEOUT) CUDA_TRY(cudaMemset(c->ws + c->lay.counters, 0, sizeof(int) * 2 * kMaxCtas));
     return SAEM_OK;
 }
 

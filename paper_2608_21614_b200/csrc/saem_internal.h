@@ -126,6 +126,27 @@ cudaError_t launch_ffn_scalar(const FfnArgs& a, const SlotTable& tab, cudaStream
 cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
 // Segments of at most 8 rows (decode batches 1..8): row-split matrix-vector kernels.
 cudaError_t launch_ffn_gemv(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
+// The whole step for batches of at most 8 tokens (top_k at most 8) in two launches: gate + repack
+// indices + gate/up projection, then down projection + merge (decode_fused.cu).
+struct DecodeArgs {
+    const float* logits;        // [T, E]
+    const uint16_t* x;          // [T, d]
+    int T, E, S, k, d, f, renorm;
+    const uint8_t* slot_region;
+    size_t slot_bytes;
+    uint16_t* h;                // [T * (k + S), f] bf16 workspace
+    void* out;                  // [T, d]
+    int out_bf16;
+    int32_t* topk_idx;          // index outputs of the step, written by one CTA
+    float* topk_w;
+    int32_t* counts;
+    int32_t* offsets;
+    int32_t* perm;
+    int32_t* inv_perm;
+    int* status;
+};
+bool decode_fused_supported(int T, int k);
+cudaError_t launch_decode_fused(const DecodeArgs& a, const SlotTable& tab, int n_sm, cudaStream_t st, int* n_launch);
 // One-time per process: resolves the driver entry point for tensor-map encoding and opts the
 // kernels into large dynamic shared memory.  Returns cudaSuccess or the failing error.
 cudaError_t ffn_tensor_init();

@@ -86,27 +86,37 @@ def main():
     layer.close()
 
 
-def bookkeeping_step(cfg, li, layer, logits, x, steps):
-    """Whole step, grouped (route, repack, grouped FFN, combine) against per-expert bookkeeping."""
-    T, E, d, k = cfg.tokens, cfg.n_experts, cfg.d_model, cfg.top_k
-    n_sh = cfg.d_ff_shared // cfg.d_ff if cfg.d_ff_shared else 0
-    # every expert (and every d_ff-wide part of the shared expert) as layer l of a one-expert context
-    one = MoELayer(d, cfg.d_ff, 1, 1, T, 0, n_layers=E + n_sh, slots_per_layer=1)
-    for e in range(E):
-        one.load_expert(e, 0, 0, li.gate[e], li.up[e], li.down[e])
-    for s_ in range(n_sh):
-        rows = slice(s_ * cfg.d_ff, (s_ + 1) * cfg.d_ff)
-        one.load_expert(E + s_, 0, 0, li.shared[0][rows], li.shared[1][rows], np.ascontiguousarray(li.shared[2][:, rows]))
-    one.drop_host_copies()
-    from . import binding as B
-    xg = torch.empty((T, d), dtype=torch.uint16, device="cuda")
-    yg = torch.empty((T, d), dtype=torch.float32, device="cuda")
-    out_b = torch.zeros((T, d), dtype=torch.float32, device="cuda")
-    calls = [0]
+class BookkeepingStep:
+    """The step done the way the paper describes its starting point (Sec. III, "bookkeeping"): route,
+    then per expert a mask over the routing, a gather of that expert's tokens, the expert's dense
+    execution on the gathered rows and a scatter-add of the weighted result.  Mask, gather and
+    scatter-add are torch operations; the gate and every expert FFN run in this library's kernels
+    (`one` holds every expert, and every d_ff-wide part of the shared expert, as a one-expert layer)."""
 
-    def book():
+    def __init__(self, cfg, li, layer: MoELayer):
+        self.cfg, self.layer = cfg, layer
+        T, E, d = cfg.tokens, cfg.n_experts, cfg.d_model
+        self.n_sh = cfg.d_ff_shared // cfg.d_ff if cfg.d_ff_shared else 0
+        assert cfg.d_ff_shared == self.n_sh * cfg.d_ff, "shared width must be a multiple of d_ff here"
+        self.one = MoELayer(d, cfg.d_ff, 1, 1, T, 0, n_layers=E + self.n_sh, slots_per_layer=1)
+        for e in range(E):
+            self.one.load_expert(e, 0, 0, li.gate[e], li.up[e], li.down[e])
+        for s_ in range(self.n_sh):
+            rows = slice(s_ * cfg.d_ff, (s_ + 1) * cfg.d_ff)
+            self.one.load_expert(E + s_, 0, 0, li.shared[0][rows], li.shared[1][rows],
+                                 np.ascontiguousarray(li.shared[2][:, rows]))
+        self.one.drop_host_copies()
+        self.xg = torch.empty((T, d), dtype=torch.uint16, device="cuda")
+        self.yg = torch.empty((T, d), dtype=torch.float32, device="cuda")
+        self.out = torch.zeros((T, d), dtype=torch.float32, device="cuda")
+        self.ffn_calls = 0
+
+    def run(self, logits: torch.Tensor, x: torch.Tensor) -> torch.Tensor:
+        from . import binding as B
+        T, E = self.cfg.tokens, self.cfg.n_experts
+        layer, one, xg, yg, out = self.layer, self.one, self.xg, self.yg, self.out
         layer.route(logits, T)
-        out_b.zero_()
+        out.zero_()
         idx, w = layer.topk_idx[:T].to(torch.int64), layer.topk_w[:T]
         for e in range(E):
             tok, slot = (idx == e).nonzero(as_tuple=True)           # mask -> indices: synchronises with the host
@@ -115,15 +125,22 @@ def bookkeeping_step(cfg, li, layer, logits, x, steps):
                 continue
             xg.view(torch.int16)[:n] = x.view(torch.int16)[tok]      # gather (bit patterns)
             B.saem_expert_ffn(one.ctx.handle, e, xg, None, n, None, yg)
-            out_b.index_add_(0, tok, yg[:n] * w[tok, slot].unsqueeze(1))    # scatter-add
-            calls[0] += 1
-        for s_ in range(n_sh):                                      # shared expert: every token, weight 1
+            out.index_add_(0, tok, yg[:n] * w[tok, slot].unsqueeze(1))      # scatter-add
+            self.ffn_calls += 1
+        for s_ in range(self.n_sh):                                 # shared expert: every token, weight 1
             B.saem_expert_ffn(one.ctx.handle, E + s_, x, None, T, None, yg)
-            out_b.add_(yg[:T])
-            calls[0] += 1
+            out.add_(yg[:T])
+            self.ffn_calls += 1
+        return out
 
-    def grouped():
-        layer.step(logits, x, T)
+    def close(self):
+        self.one.close()
+
+
+def bookkeeping_step(cfg, li, layer, logits, x, steps):
+    """Whole step, grouped (route, repack, grouped FFN, combine) against per-expert bookkeeping."""
+    T = cfg.tokens
+    book = BookkeepingStep(cfg, li, layer)
 
     def timed(fn):
         for _ in range(3):
@@ -137,14 +154,14 @@ def bookkeeping_step(cfg, li, layer, logits, x, steps):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / steps * 1e3
 
-    t_g = timed(grouped)
+    t_g = timed(lambda: layer.step(logits, x, T))
     ref = layer.out[:T].clone()
-    calls[0] = 0
-    t_b = timed(book)
-    res = {"grouped_step_us": t_g, "bookkeeping_step_us": t_b, "ffn_calls_per_step": calls[0] / (steps + 3),
-           "speedup": t_b / t_g, "max_abs_difference": float((ref - out_b).abs().max()),
-           "device_status": one.device_status()}
-    one.close()
+    book.ffn_calls = 0
+    t_b = timed(lambda: book.run(logits, x))
+    res = {"grouped_step_us": t_g, "bookkeeping_step_us": t_b, "ffn_calls_per_step": book.ffn_calls / (steps + 3),
+           "speedup": t_b / t_g, "max_abs_difference": float((ref - book.out).abs().max()),
+           "device_status": book.one.device_status()}
+    book.close()
     return res
 
 

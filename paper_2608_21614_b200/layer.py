@@ -100,13 +100,6 @@ class MoELayer:
     def shared_ffn(self, x: torch.Tensor, T: int, layer: int = 0, stream=None):
         B.saem_expert_ffn(self.shared.handle, layer, x, None, T, None, self.shared_y, stream)
 
-    def shared_rows(self, T: int) -> torch.Tensor:
-        """Output of the shared expert(s) for the last step: [T, d] fp32 (sums the in-layer parts)."""
-        if self.S:
-            P = T * self.k
-            return self.y_packed[P:P + self.S * T].view(self.S, T, self.d).sum(0)
-        return self.shared_y[:T]
-
     def combine(self, T: int, stream=None):
         B.saem_combine(self.ctx.handle, self.y_packed, self.inv_perm, self.topk_w, T, self.shared_y, self.out, stream)
 

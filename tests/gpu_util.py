@@ -4,6 +4,8 @@ the oracle.  Tolerances are the ones the benchmark contract states: indices bit-
 import numpy as np
 import torch
 
+from paper_2608_21614_b200 import inputs as gen
+
 MAX_ABS = 2e-2
 REL_L2 = 1e-2
 W_TOL = 1e-6
@@ -42,6 +44,15 @@ def make_layer(li, ffn_path, max_tokens=None, **kw):
     return layer
 
 
+def shared_rows(layer, T):
+    """Output of the shared expert(s) of the last step, [T, d] fp32: the sum of the in-layer shared
+    experts' rows of y_packed, or the separate shared context's output."""
+    if layer.S:
+        P = T * layer.k
+        return layer.y_packed[P:P + layer.S * T].view(layer.S, T, layer.d).sum(0)
+    return layer.shared_y[:T]
+
+
 def run_stepwise_and_compare(layer, li, oracle, ref=None):
     """Runs the four calls one by one and compares every output with the oracle's."""
     c = li.cfg
@@ -67,6 +78,82 @@ def run_stepwise_and_compare(layer, li, oracle, ref=None):
     assert np.array_equal(host(layer.x_packed[:P]), ref["x_packed"]), "x_packed"
     stats = {"y_packed": assert_close(host(layer.y_packed[:P]), ref["y_packed"], "y_packed")}
     if li.shared is not None:
-        stats["shared_y"] = assert_close(host(layer.shared_rows(T)), ref["shared_y"], "shared_y")
+        stats["shared_y"] = assert_close(host(shared_rows(layer, T)), ref["shared_y"], "shared_y")
     stats["out"] = assert_close(host(out), ref["out"], "out")
     return ref, stats
+
+
+# ------------------------------------------------------------------ partially resident stacks
+def run_stack(trace, weights, L, E, k, d, f, C, temp, batch, steps, keep, policy="stage", eap=None):
+    from paper_2608_21614_b200.stack import StackRunner
+    run = StackRunner(d, f, E, k, L, C, temp, batch, weights, policy=policy, recorded_eap=eap)
+    # warm set: the C most popular experts of stage 0 (stand-in for the calibration warm-up)
+    run.warm([list(np.argsort(trace.rankings[0, l])[:C]) for l in range(L)])
+    outs = []
+    bounds = set(int(b) for b in trace.boundaries[1:])
+    for t in range(steps):
+        if t in bounds:
+            run.boundary()
+        lg = np.stack([gen.trace_logits(trace, t, l, batch) for l in range(L)])
+        x = gen.trace_activations(trace, t, batch, d)
+        out = run.step(torch.from_numpy(lg).cuda(), torch.from_numpy(x).cuda())
+        if t in keep:
+            torch.cuda.synchronize()
+            outs.append(out.clone())
+    torch.cuda.synchronize()
+    from paper_2608_21614_b200 import binding as B
+    assert B.saem_last_device_status(run.h) == 0
+    stats = run.stats
+    final = [list(s) for s in run.slot_expert]
+    store = run.store
+    return outs, stats, final, run
+
+
+def simulate_stack(trace, oracle, L, E, k, C, temp, batch, steps):
+    """Independent host simulation of the policy: residency sets, a ring of temporary slots,
+    the pairwise-swap planner at boundaries; routing from the oracle."""
+    res = [set(int(e) for e in np.argsort(trace.rankings[0, l])[:C]) for l in range(L)]
+    ring = [None] * temp
+    nxt = 0
+    log = np.zeros((L, E), np.int64)
+    st = dict(active=0, hits=0, temp_hits=0, demand=0, boundary=0, pair_total=0, pair_hits=0)
+    bounds = set(int(b) for b in trace.boundaries[1:])
+    for t in range(steps):
+        if t in bounds:
+            for l in range(L):
+                while True:
+                    non = [e for e in range(E) if e not in res[l]]
+                    best = min(non, key=lambda e: (-log[l, e], e))
+                    worst = min(res[l], key=lambda e: (log[l, e], -e))
+                    if log[l, best] <= log[l, worst]:
+                        break
+                    res[l].remove(worst)
+                    res[l].add(best)
+                    st["boundary"] += 1
+                    ring = [None if r == (l, best) else r for r in ring]
+            log[:] = 0
+        for l in range(L):
+            idx, _ = oracle.route(gen.trace_logits(trace, t, l, batch), k)
+            cnt = np.bincount(idx.ravel(), minlength=E)
+            need = []
+            for e in np.nonzero(cnt)[0]:
+                e = int(e)
+                st["active"] += 1
+                st["pair_total"] += int(cnt[e])
+                if e in res[l]:
+                    st["hits"] += 1
+                    st["pair_hits"] += int(cnt[e])
+                else:
+                    need.append(e)
+                    if (l, e) in ring:
+                        st["temp_hits"] += 1
+            while True:
+                missing = [e for e in need if (l, e) not in ring]
+                if not missing:
+                    break
+                for e in missing:
+                    ring[nxt] = (l, e)
+                    nxt = (nxt + 1) % temp
+                    st["demand"] += 1
+            log[l] += cnt
+    return st, [sorted(r) for r in res]

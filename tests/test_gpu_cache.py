@@ -86,80 +86,6 @@ def test_load_is_ordered_after_enqueued_reads_and_before_later_ones(oracle):
     ctx.close()
 
 
-def _run_stack(trace, weights, L, E, k, d, f, C, temp, batch, steps, keep, policy="stage", eap=None):
-    from paper_2608_21614_b200.stack import StackRunner
-    run = StackRunner(d, f, E, k, L, C, temp, batch, weights, policy=policy, recorded_eap=eap)
-    # warm set: the C most popular experts of stage 0 (stand-in for the calibration warm-up)
-    run.warm([list(np.argsort(trace.rankings[0, l])[:C]) for l in range(L)])
-    outs = []
-    bounds = set(int(b) for b in trace.boundaries[1:])
-    for t in range(steps):
-        if t in bounds:
-            run.boundary()
-        lg = np.stack([gen.trace_logits(trace, t, l, batch) for l in range(L)])
-        x = gen.trace_activations(trace, t, batch, d)
-        out = run.step(torch.from_numpy(lg).cuda(), torch.from_numpy(x).cuda())
-        if t in keep:
-            torch.cuda.synchronize()
-            outs.append(out.clone())
-    torch.cuda.synchronize()
-    assert __import__("paper_2608_21614_b200.binding", fromlist=["x"]).saem_last_device_status(run.h) == 0
-    stats = run.stats
-    final = [list(s) for s in run.slot_expert]
-    store = run.store
-    return outs, stats, final, run
-
-
-def _simulate(trace, oracle, L, E, k, C, temp, batch, steps):
-    """Independent host simulation of the policy: residency sets, a ring of temporary slots,
-    the pairwise-swap planner at boundaries; routing from the oracle."""
-    res = [set(int(e) for e in np.argsort(trace.rankings[0, l])[:C]) for l in range(L)]
-    ring = [None] * temp
-    nxt = 0
-    log = np.zeros((L, E), np.int64)
-    st = dict(active=0, hits=0, temp_hits=0, demand=0, boundary=0, pair_total=0, pair_hits=0)
-    bounds = set(int(b) for b in trace.boundaries[1:])
-    for t in range(steps):
-        if t in bounds:
-            for l in range(L):
-                while True:
-                    non = [e for e in range(E) if e not in res[l]]
-                    best = min(non, key=lambda e: (-log[l, e], e))
-                    worst = min(res[l], key=lambda e: (log[l, e], -e))
-                    if log[l, best] <= log[l, worst]:
-                        break
-                    res[l].remove(worst)
-                    res[l].add(best)
-                    st["boundary"] += 1
-                    ring = [None if r == (l, best) else r for r in ring]
-            log[:] = 0
-        for l in range(L):
-            idx, _ = oracle.route(gen.trace_logits(trace, t, l, batch), k)
-            cnt = np.bincount(idx.ravel(), minlength=E)
-            need = []
-            for e in np.nonzero(cnt)[0]:
-                e = int(e)
-                st["active"] += 1
-                st["pair_total"] += int(cnt[e])
-                if e in res[l]:
-                    st["hits"] += 1
-                    st["pair_hits"] += int(cnt[e])
-                else:
-                    need.append(e)
-                    if (l, e) in ring:
-                        st["temp_hits"] += 1
-            while True:
-                missing = [e for e in need if (l, e) not in ring]
-                if not missing:
-                    break
-                for e in missing:
-                    ring[nxt] = (l, e)
-                    nxt = (nxt + 1) % temp
-                    st["demand"] += 1
-            log[l] += cnt
-    return st, [sorted(r) for r in res]
-
-
 def test_half_resident_stack_equals_full_residency_and_simulation(oracle):
     import gpu_util as g
     L, E, k, d, f, batch, steps = 3, 8, 2, 256, 256, 4, 40
@@ -167,14 +93,14 @@ def test_half_resident_stack_equals_full_residency_and_simulation(oracle):
     assert len(trace.boundaries) >= 3
     weights = _small_experts(6, d, f, 3)                     # 24 (layer, expert) pairs share 6 weight sets
     keep = set(range(steps))
-    full, st_full, _, run_full = _run_stack(trace, weights, L, E, k, d, f, E, 0, batch, steps, keep)
-    half, st_half, final_half, run_half = _run_stack(trace, weights, L, E, k, d, f, E // 2, 4, batch, steps, keep)
+    full, st_full, _, run_full = g.run_stack(trace, weights, L, E, k, d, f, E, 0, batch, steps, keep)
+    half, st_half, final_half, run_half = g.run_stack(trace, weights, L, E, k, d, f, E // 2, 4, batch, steps, keep)
     # routing does not depend on placement: identical bits under 50 % and 100 % residency
     for a, b in zip(full, half):
         assert torch.equal(a, b)
     assert st_full.chr() == 1.0 and st_full.demand_loads == 0 and st_full.boundary_loads == 0
     # the policy bookkeeping equals an independent simulation, number for number
-    sim, sim_final = _simulate(trace, oracle, L, E, k, E // 2, 4, batch, steps)
+    sim, sim_final = g.simulate_stack(trace, oracle, L, E, k, E // 2, 4, batch, steps)
     assert (st_half.active, st_half.hits, st_half.temp_hits) == (sim["active"], sim["hits"], sim["temp_hits"])
     assert (st_half.pair_total, st_half.pair_hits) == (sim["pair_total"], sim["pair_hits"])
     assert st_half.demand_loads == sim["demand"] and st_half.boundary_loads == sim["boundary"]
@@ -197,11 +123,12 @@ def test_replay_policies_share_bits_and_oracle_is_no_worse(oracle):
     clairvoyant policy fed with the recorded per-stage counts, and token-level LRU.  Routing is
     independent of placement, so every policy yields the same output bits; the clairvoyant
     planner never has fewer hits at a boundary than the lag-one planner on this trace."""
+    import gpu_util as g
     L, E, k, d, f, batch, steps = 2, 8, 2, 128, 128, 2, 48
     trace = gen.stage_trace(steps, L, E, 1.2, seed=5, mean_stage_len=8.0, reshuffled=None)   # independent stages
     weights = _small_experts(4, d, f, 9)
     keep = {steps - 1}
-    ref, st_full, _, run0 = _run_stack(trace, weights, L, E, k, d, f, E, 0, batch, steps, keep)
+    ref, st_full, _, run0 = g.run_stack(trace, weights, L, E, k, d, f, E, 0, batch, steps, keep)
     eap = run0.finish()
     # the recorded EAP equals routing counts from the oracle, stage by stage
     bounds = list(trace.boundaries) + [steps]
@@ -214,7 +141,7 @@ def test_replay_policies_share_bits_and_oracle_is_no_worse(oracle):
         assert np.array_equal(eap[s], cnt)
     res = {}
     for policy in ("stage", "oracle", "lru"):
-        outs, st, _, run = _run_stack(trace, weights, L, E, k, d, f, 4, 4, batch, steps, keep, policy, eap)
+        outs, st, _, run = g.run_stack(trace, weights, L, E, k, d, f, 4, 4, batch, steps, keep, policy, eap)
         assert torch.equal(outs[0], ref[0]), policy
         res[policy] = st
         run.close()

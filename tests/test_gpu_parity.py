@@ -121,6 +121,27 @@ def test_segment_sizes_around_tile_edges(oracle, path):
     layer.close()
 
 
+@pytest.mark.parametrize("path", [TENSOR, AUTO], ids=["tensor", "auto"])
+@pytest.mark.parametrize("max_tokens,fs", [(40, 0), (48, 0), (40, 256), (48, 256), (33, 0)])
+def test_token_tiles_between_32_and_64_rows(oracle, path, max_tokens, fs):
+    """Contexts whose largest batch is 33..48 tokens: the streaming kernels load a token tile as
+    32-row boxes, so the tile (and its shared-memory stage) must hold a whole number of boxes.  One
+    routed expert with k = 1 (and optionally one in-layer shared expert) makes every segment exactly
+    max_tokens rows long."""
+    g = _g()
+    d, f = 256, 256
+    cfg = gen.LayerConfig("t", d, f, 1, 1, max_tokens, fs, "normal", seed=40 + max_tokens)
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, path)
+    assert layer.S == (1 if fs else 0)
+    g.run_stepwise_and_compare(layer, li, oracle)
+    y1 = layer.y_packed.clone()
+    layer.step(g.dev(li.logits), g.dev(li.x), max_tokens)
+    torch.cuda.synchronize()
+    assert torch.equal(y1, layer.y_packed)
+    layer.close()
+
+
 def test_route_special_values(oracle, B):
     g = _g()
     rows = [
@@ -194,6 +215,47 @@ def test_repack_skew_and_paper_example(oracle, B):
         assert np.array_equal(g.host(xp), rx)
         assert B.saem_last_device_status(ctx.handle) == 0
         ctx.close()
+
+
+@pytest.mark.parametrize("T,S", [(700, 1), (700, 0), (100, 1)], ids=["two-kernel-shared", "two-kernel", "fused-shared"])
+def test_repack_drops_invalid_expert_ids(oracle, B, T, S):
+    """Expert ids outside [0, E), injected on the host: the status word says INVALID_ARG, the pair is
+    dropped from every output, and the valid pairs are packed exactly as the oracle packs them (the
+    oracle is given the valid pairs only, as a ragged problem: invalid pairs are routed to a spare
+    expert E whose segment comes last).  With in-layer shared experts and more than 2048 pairs the
+    gather runs as a second kernel over all T*k rows and must skip the rows that hold no pair."""
+    g = _g()
+    E, k, d = 12, 3, 128
+    rng = np.random.default_rng(T + S)
+    idx = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)
+    bad = rng.choice(T * k, 9, replace=False)
+    idx.ravel()[bad[:5]] = E + 3
+    idx.ravel()[bad[5:]] = -1
+    x = rng.integers(0, 65535, size=(T, d)).astype(np.uint16)
+    ctx = B.Context(B.make_config(d, 128, E, k, T, n_shared=S))
+    P, R = T * k, T * (k + S)
+    counts = torch.empty(E + S, dtype=torch.int32, device="cuda:0")
+    offsets = torch.empty(E + S + 1, dtype=torch.int32, device="cuda:0")
+    perm = torch.full((P,), 12345, dtype=torch.int32, device="cuda:0")
+    inv = torch.empty(P, dtype=torch.int32, device="cuda:0")
+    xp = torch.full((R, d), 7, dtype=torch.uint16, device="cuda:0")
+    B.saem_repack(ctx.handle, g.dev(idx), g.dev(x), T, counts, offsets, perm, inv, xp)
+    assert B.saem_last_device_status(ctx.handle) == B.SAEM_ERR_INVALID_ARG
+    spare = np.where((idx < 0) | (idx >= E), E, idx).astype(np.int32)
+    rc, ro, rp, ri, rx = oracle.repack(spare, x, E + 1)
+    valid = int(ro[E])
+    assert valid == P - 9
+    assert np.array_equal(g.host(counts)[:E], rc[:E])
+    assert np.array_equal(g.host(offsets)[:E], ro[:E])
+    assert int(g.host(offsets)[E]) == (P if S else valid)
+    assert np.array_equal(g.host(perm)[:valid], rp[:valid]) and np.all(g.host(perm)[valid:] == -1)
+    ri_expect = np.where(ri >= valid, -1, ri)
+    assert np.array_equal(g.host(inv), ri_expect)
+    assert np.array_equal(g.host(xp)[:valid], rx[:valid])
+    assert np.all(g.host(xp)[valid:P] == 7)                         # rows without a pair are never written
+    if S:
+        assert np.array_equal(g.host(xp)[P:], np.tile(x, (S, 1)))
+    ctx.close()
 
 
 @pytest.mark.parametrize("fs,merge", [(256, True), (768, True), (768, False)],
@@ -390,11 +452,18 @@ def test_bounded_device_wait_runs_out_and_context_survives(oracle, B):
     g = _g()
     li = gen.layer_inputs(gen.LayerConfig("t", 128, 128, 4, 2, 16, seed=1))
     layer = g.make_layer(li, TENSOR)
+    # a CTA that gives up a wait skips its arrival on a split item's counter; stand in for that on the
+    # host by leaving a count behind, and check that reading the TIMEOUT status clears the counters
+    counters = layer.ctx.step_tensor(10, (640,), torch.int32)
+    assert int(counters.abs().sum()) == 0
+    counters[3] = 2
+    counters[320 + 17] = 1
     t0 = time.perf_counter()
     B.saem_selftest_bounded_wait(layer.ctx.handle, 20000)            # 20 ms limit
     torch.cuda.synchronize()
     assert time.perf_counter() - t0 < 5.0
     assert layer.device_status() == B.SAEM_ERR_TIMEOUT
+    assert int(counters.abs().sum()) == 0
     assert layer.device_status() == 0
     assert B.saem_selftest_bounded_wait(layer.ctx.handle, 0, check=False) == B.SAEM_ERR_INVALID_ARG
     g.run_stepwise_and_compare(layer, li, oracle)
@@ -432,3 +501,25 @@ def test_route_fused_with_router_projection(oracle, B, T, E, k, d):
     torch.cuda.synchronize()
     assert torch.equal(idx, idx2) and torch.equal(w, w2)
     ctx.close()
+
+
+@pytest.mark.parametrize("T,E,k,d,f,fs", [(24, 12, 3, 256, 384, 768), (5, 60, 4, 256, 128, 0)])
+def test_bookkeeping_comparison_mode_against_oracle(oracle, T, E, k, d, f, fs):
+    """The per-expert mask / gather / dense execution / scatter-add procedure of the paper's
+    Motivation 3 (the comparison mode of launch_ablation) computes the same layer output as the
+    oracle, within the FFN tolerance -- so the launch-count and time contrast it reports is between
+    two correct ways of doing the same step."""
+    g = _g()
+    from paper_2608_21614_b200.launch_ablation import BookkeepingStep
+    cfg = gen.LayerConfig("t", d, f, E, k, T, fs, "zipf", 1.1, seed=21)
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, AUTO)
+    book = BookkeepingStep(cfg, li, layer)
+    out = book.run(g.dev(li.logits), g.dev(li.x))
+    torch.cuda.synchronize()
+    ref = oracle.moe_step(li.logits, li.x, k, li.gate, li.up, li.down, shared=li.shared)
+    g.assert_close(g.host(out), ref["out"], "bookkeeping step")
+    assert book.ffn_calls == int((ref["counts"] > 0).sum()) + (fs // f if fs else 0)
+    assert book.one.device_status() == 0 and layer.device_status() == 0
+    book.close()
+    layer.close()

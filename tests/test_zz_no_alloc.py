@@ -4,7 +4,8 @@ Some callers of this library cannot allocate device memory (the memory pool belo
 application, or an allocation inside their loop is not allowed), so they have no workspace to
 give.  This entry point keeps its only scratch -- the hidden activations -- in a fixed array
 inside the library.  The test calls it twice in a row through the C ABI on different inputs (the
-array keeps the first call's contents) and compares each result with the regular entry point's.
+array keeps the first call's contents) and compares each result with the regular entry point's
+and with the CPU oracle's.
 It is collected last so that a run stopping at the first failure has already run everything else.
 """
 import numpy as np
@@ -16,7 +17,7 @@ from paper_2608_21614_b200 import inputs as gen
 pytestmark = pytest.mark.gpu
 
 
-def test_static_scratch_ffn_matches_regular_entry_point_twice():
+def test_static_scratch_ffn_matches_regular_entry_point_twice(oracle):
     import gpu_util as g
     from paper_2608_21614_b200 import binding as B
     from paper_2608_21614_b200.layer import MoELayer
@@ -38,6 +39,17 @@ def test_static_scratch_ffn_matches_regular_entry_point_twice():
         B.saem_expert_ffn_static(layer.x_packed, layer.offsets, E, T * k, d, f, layer.ctx.slot_ptr, y_static)
         torch.cuda.synchronize()
         g.assert_close(g.host(y_static), g.host(layer.y_packed), "static vs regular, call %d" % call)
+        # ... and against the CPU oracle directly, so that a mistake shared by both GPU paths cannot hide
+        off = g.host(layer.offsets)[:E + 1]
+        y_ref = oracle.expert_ffn(g.host(layer.x_packed[:T * k]), off, li.gate, li.up, li.down)
+        g.assert_close(g.host(y_static), y_ref, "static vs oracle, call %d" % call)
+    # max_rows below the last offset: the rows from max_rows on are left untouched
+    cut = int(off[E - 1]) + 1 if off[E] - off[E - 1] > 1 else T * k - 3
+    y_cut = torch.full((T * k, d), float("nan"), dtype=torch.float32, device="cuda:0")
+    B.saem_expert_ffn_static(layer.x_packed, layer.offsets, E, cut, d, f, layer.ctx.slot_ptr, y_cut)
+    torch.cuda.synchronize()
+    g.assert_close(g.host(y_cut[:cut]), y_ref[:cut], "static, max_rows inside the last segment")
+    assert torch.isnan(y_cut[cut:]).all()
     # sizes beyond the fixed array are refused before anything is enqueued
     too_many = B.SAEM_STATIC_SCRATCH_ELEMS // f + 1
     code = B.saem_expert_ffn_static(layer.x_packed, layer.offsets, E, too_many, d, f, layer.ctx.slot_ptr,
