@@ -61,7 +61,7 @@ typedef enum saem_status {
 enum { SAEM_MAX_EXPERTS = 128 };         /* routed experts per layer */
 enum { SAEM_TEMP = -2 };                 /* slot argument of saem_cache_load: take a temporary slot */
 enum { SAEM_OUT_F32 = 0, SAEM_OUT_BF16 = 1 };
-enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TENSOR_PAIRS = 3 };
+enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TENSOR_PAIRS = 3, SAEM_FFN_DECODE_FUSED = 4 };
 
 /*
  * Shape of one context.  d_model and d_ff must be multiples of 128, at most 16384; 1 <= top_k <= n_experts <=
@@ -77,7 +77,9 @@ enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TEN
  * (tcgen05 cta_group::2: 256 tokens x 512 weight rows per pair of SMs), which AUTO and TENSOR take
  * for long reductions and many rows (d_model >= 4096, d_model % 256 == 0, at least 1536 packed
  * rows in the call); SAEM_FFN_TENSOR_PAIRS is SAEM_FFN_TENSOR with the pair form whenever
- * d_model % 256 == 0 (for tests and measurements).
+ * d_model % 256 == 0 (for tests and measurements).  SAEM_FFN_DECODE_FUSED is SAEM_FFN_AUTO, except that
+ * saem_moe_step takes its one-launch form (see there) for every batch it supports (up to 8 tokens, top_k
+ * up to 8) instead of up to 4 tokens.
  * n_shared (0..16, n_experts + n_shared <= SAEM_MAX_EXPERTS): always-on shared experts of the same
  * width d_ff that run INSIDE the layer's grouped launch.  They are experts n_experts ..
  * n_experts + n_shared - 1 of every layer for the cache calls (outside the routed cache-ratio
@@ -210,6 +212,12 @@ int saem_combine(saem_ctx* ctx, const float* y_packed, const int32_t* inv_perm, 
  * holds an always-on shared expert whose width is not a multiple of d_ff (otherwise use
  * config.n_shared and pass NULL).
  * logits[T, E] fp32, x[T, d] bf16, out[T, d] (all dev).
+ * Smallest decode batches (ffn_path AUTO: T <= 4; top_k <= 8; no shared_ctx): the whole step runs as ONE
+ * kernel launch -- gate, repack indices and gate/up projection, a grid-wide barrier, down projection and
+ * merge -- launched cooperatively (two launches where the device refuses that).  topk_idx, topk_w, counts,
+ * offsets, perm, inv_perm, h and y_packed are still left in the workspace; x_packed is not produced.  A
+ * routed expert without a slot sets NOT_RESIDENT in the device status word and contributes nothing.  The
+ * first such call on a device should come before any stream capture (it probes what the driver accepts).
  */
 int saem_moe_step(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const float* logits, const void* x, int T,
                   void* out, void* stream);

@@ -21,7 +21,7 @@ SAEM_ERR_NOT_RESIDENT, SAEM_ERR_SLOT_BUSY, SAEM_ERR_TIMEOUT, SAEM_ERR_CUDA, SAEM
 SAEM_MAX_EXPERTS = 128
 SAEM_TEMP = -2
 SAEM_OUT_F32, SAEM_OUT_BF16 = 0, 1
-SAEM_FFN_AUTO, SAEM_FFN_SCALAR, SAEM_FFN_TENSOR, SAEM_FFN_TENSOR_PAIRS = 0, 1, 2, 3
+SAEM_FFN_AUTO, SAEM_FFN_SCALAR, SAEM_FFN_TENSOR, SAEM_FFN_TENSOR_PAIRS, SAEM_FFN_DECODE_FUSED = 0, 1, 2, 3, 4
 
 
 class saem_config(C.Structure):

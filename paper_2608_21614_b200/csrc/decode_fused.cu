@@ -1,44 +1,54 @@
-// The whole MoE layer step for the smallest decode batches (at most 8 tokens, top-k at most 8) in
-// two launches instead of five.  At batch 1-8 the step moves a few tens of megabytes, so a launch's
-// fixed cost (start-up, finding the active experts, the last partial wave) is as large as its
-// streaming time; the paper's operating point is exactly this regime (batch 1-8 decode).
+// The whole MoE layer step for the smallest decode batches (at most 8 tokens, top-k at most 8) in ONE
+// launch instead of five.  At batch 1-8 the step moves a few tens of megabytes, so a launch's fixed
+// cost (start-up, finding the active experts, the last partial wave) is as large as its streaming
+// time; the paper's operating point is exactly this regime (batch 1-8 decode).
 //
-//   decode_gateup_kernel        every CTA repeats the tiny gate (top-k of E logits for <= 8 tokens,
-//                               Background "Mixture-of-Experts Inference") and the expert-aligned
-//                               repack indices (Sec. IV-E: counts, exclusive scan, stable
-//                               permutation) in its own shared memory, then streams its share of the
-//                               ACTIVE experts' gate/up rows and writes h = silu(Wg x) * (Wu x).
-//                               Token rows are read straight from x through the permutation: no
-//                               x_packed round trip.  CTA 0 also writes the index outputs, so they
-//                               stay inspectable and bit-exact.
-//   decode_down_combine_kernel  a CTA owns 16 output columns for ALL active experts: it streams those
-//                               16 rows of every active expert's down matrix, keeps the per-pair
-//                               results in shared memory and merges them per token in slot order
-//                               j = 0..k-1, shared experts last (Sec. IV-D merge; deterministic, no
-//                               atomics): no y_packed round trip and no combine launch.  It repeats
-//                               the gate from the logits itself and starts streaming weights BEFORE
-//                               it waits for the first kernel (programmatic dependent launch), so its
-//                               start-up hides behind the first kernel's tail.
+// One persistent CTA per SM, 16 warps.  Every CTA repeats the tiny gate (top-k of E logits for <= 8
+// tokens; Background "Mixture-of-Experts Inference") and the expert-aligned repack indices (Sec. IV-E:
+// counts, exclusive scan, stable permutation) in its own shared memory -- CTA 0 also writes them out,
+// so they stay inspectable and bit-exact -- and then the grid runs two streaming phases:
 //
-// Both kernels are shaped by bytes (decode is weight streaming): 16-byte loads of the packed slot
-// layout's 128-byte tile rows, mma.sync m16n8k16 as the arithmetic unit (16 weight rows x up to 8
-// tokens), fp32 accumulation, fixed summation orders.  The second kernel keeps a deep queue of loads
-// in flight without spending registers on it: every warp owns a ring of shared-memory stages that
-// its lanes fill with cp.async (each lane copies exactly the bytes its own MMA fragments need, so no
-// barrier is involved), because with one CTA per 16 output columns there are only d_model / 16 CTAs.
+//   phase A  h = silu(Wg x) * (Wu x).  A warp's unit is 16 hidden units of one ACTIVE expert over the
+//            whole reduction length: an MMA's 16 rows are 8 gate rows and the 8 matching up rows, so
+//            SiLU*mul happens in the accumulator registers of one thread and nothing is exchanged
+//            between warps.  Token rows are read straight from x through the permutation (no x_packed).
+//   phase B  y = Wd h for 32 output columns of one active expert per warp unit, then the merge (Sec.
+//            IV-D): each group of 32 columns has a ticket counter, and the warp that delivers a
+//            group's last expert adds the k contributions of every token in slot order j = 0..k-1,
+//            shared experts last, with the arithmetic of the combine kernel (deterministic whoever
+//            does it; nobody waits for anybody).
+//
+// Between the phases the grid meets at a barrier (a cooperative launch guarantees that all CTAs are
+// resident; the wait is bounded and gives up with SAEM_ERR_TIMEOUT).  Before it arrives, every warp
+// has already requested the first weight stages of its phase-B unit, so the barrier and the L2 round
+// trip of h hide behind loads in flight.  Where a cooperative launch is not available the same kernel
+// runs as two launches (phase A, phase B), the second waiting for the first by programmatic dependent
+// launch after it has requested its first weights.
+//
+// Shaped by bytes (decode is weight streaming): a chunk of a unit is 4 KB of consecutive rows of the
+// packed slot layout's tiles, fetched by one cp.async.bulk into the warp's own ring of shared-memory
+// stages (three in flight per warp, 192 KB per SM, no registers spent on loads in flight; 16-byte
+// cp.async per lane was tried first and was bound by the SM's memory-instruction queue);
+// mma.sync m16n8k16 is the arithmetic unit (16 weight rows x up to 8 tokens, fp32 accumulation),
+// reading the XOR-swizzled rows without bank conflicts; activation pieces come from L1 / L2 into
+// registers one chunk ahead.  Every warp gets one contiguous range of k-chunks; when a range cuts a
+// unit, the partial tiles are added in warp order through shared memory.
 #include <cuda_bf16.h>
 
 #include "route_row.cuh"
+#include "tc_common.cuh"
 
 namespace saem {
 
 constexpr int kDfMaxTokens = 8;
 constexpr int kDfMaxK = 8;
 constexpr int kDfMaxPairs = kDfMaxTokens * kDfMaxK;
-constexpr int kDfMaxRows = kDfMaxTokens * (kDfMaxK + 16);      // pair rows, then T rows per shared expert
-constexpr int kDfThreadsA = 256;
-constexpr int kDfWarpsA = kDfThreadsA / 32;
-constexpr int kDfRows = 16;                                    // weight rows per MMA
+constexpr int kDfWarps = 16;
+constexpr int kDfThreads = kDfWarps * 32;
+constexpr int kDfStages = 3;
+constexpr int kDfStageBytes = 4096;              // per warp and stage: the 32 weight rows of one chunk of a unit
+constexpr int kDfRingBytes = kDfWarps * kDfStages * kDfStageBytes + 128;
+constexpr unsigned long long kDfBarrierLimitNs = 200000000ull;   // 0.2 s
 
 struct DecodeIndex {
     int32_t idx[kDfMaxPairs];
@@ -47,8 +57,10 @@ struct DecodeIndex {
     int32_t inv[kDfMaxPairs];
     int32_t counts[SAEM_MAX_EXPERTS];
     int32_t offsets[SAEM_MAX_EXPERTS + 1];
-    int16_t act[SAEM_MAX_EXPERTS];          // experts with rows, ascending id
+    int16_t act[SAEM_MAX_EXPERTS];          // experts with rows AND a slot, ascending id
+    int warp_act[4];
     int n_active;
+    int absent;                             // an expert with rows has no slot
 };
 
 __device__ __forceinline__ void mma_16816(float* c, const uint32_t a0, const uint32_t a1, const uint32_t a2,
@@ -58,46 +70,59 @@ __device__ __forceinline__ void mma_16816(float* c, const uint32_t a0, const uin
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
-// Gate and repack indices of the whole (tiny) batch in shared memory; every thread of the CTA calls
-// it (at least 8 warps).  Same arithmetic and tie rules as route_kernel / the repack kernels: slots
-// in descending logit order, segments in ascending expert id, ascending pair id inside a segment,
-// one segment of all T tokens per in-layer shared expert behind the T*k pair rows.
-__device__ __forceinline__ void build_index(const DecodeArgs& a, DecodeIndex& sm) {
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+// Activation pieces come through L1: the 16 warps of a CTA read the same few token rows over and over (x is an
+// input; h is first touched by this CTA after the grid barrier, so no stale line can be in L1).
+__device__ __forceinline__ uint4 ld_act(const uint16_t* p) {
+    uint4 v;
+    asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+// Gate and repack indices of the whole (tiny) batch in shared memory; every thread of the CTA calls it.
+// Same arithmetic and tie rules as route_kernel / the repack kernels: slots in descending logit order,
+// segments in ascending expert id, ascending pair id inside a segment, one segment of all T tokens per
+// in-layer shared expert behind the T*k pair rows.  counts[e] = #{p: idx[p] == e} and offsets[e] =
+// #{p: idx[p] < e} come from one sweep over the (at most 64) pairs: no scan is needed.
+__device__ __forceinline__ void build_index(const DecodeArgs& a, const SlotTable& tab, DecodeIndex& sm) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int P = a.T * a.k, ES = a.E + a.S;
     if (warp < a.T)
         route_row(a.logits + (size_t)warp * a.E, a.E, a.k, a.renorm, lane, &sm.idx[warp * a.k], &sm.w[warp * a.k]);
+    if (tid == 0) sm.absent = 0;
     __syncthreads();
-    if (tid < ES) {
-        int c = a.T;
+    if (tid < SAEM_MAX_EXPERTS) {                     // four whole warps: the ballots below need them
+        int c = 0, o = 0;
         if (tid < a.E) {
-            c = 0;
-            for (int p = 0; p < P; ++p) c += sm.idx[p] == tid ? 1 : 0;
-        }
-        sm.counts[tid] = c;
-    }
-    __syncthreads();
-    if (warp == 0) {
-        int carry = 0, carry_act = 0;
-        for (int base = 0; base < ES; base += 32) {
-            const int e = base + lane;
-            const int v = e < ES ? sm.counts[e] : 0;
-            int inc = v;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int n = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc += n;
+            for (int p = 0; p < P; ++p) {
+                const int e = sm.idx[p];
+                c += e == tid ? 1 : 0;
+                o += e < tid ? 1 : 0;
             }
-            const unsigned actm = __ballot_sync(0xffffffffu, v > 0);
-            if (e < ES) sm.offsets[e] = carry + inc - v;
-            if (v > 0) sm.act[carry_act + __popc(actm & ((1u << lane) - 1u))] = (int16_t)e;
-            carry += __shfl_sync(0xffffffffu, inc, 31);
-            carry_act += __popc(actm);
+        } else if (tid < ES) {
+            c = a.T;
+            o = P + (tid - a.E) * a.T;
         }
-        if (lane == 0) { sm.offsets[ES] = carry; sm.n_active = carry_act; }
+        if (tid < ES) { sm.counts[tid] = c; sm.offsets[tid] = o; }
+        if (tid == ES) sm.offsets[ES] = P + a.S * a.T;
+        const bool has_rows = tid < ES && c > 0;
+        if (has_rows && tab.slot[tid] < 0) sm.absent = 1;
+        const unsigned actm = __ballot_sync(0xffffffffu, has_rows && tab.slot[tid] >= 0);
+        if (lane == 0) sm.warp_act[warp] = __popc(actm);
     }
+    if (tid == SAEM_MAX_EXPERTS && ES == SAEM_MAX_EXPERTS) sm.offsets[ES] = P + a.S * a.T;
     __syncthreads();
+    if (tid < SAEM_MAX_EXPERTS) {
+        const bool act = tid < ES && sm.counts[tid] > 0 && tab.slot[tid] >= 0;
+        const unsigned actm = __ballot_sync(0xffffffffu, act);
+        int before = __popc(actm & ((1u << lane) - 1u));
+        for (int w = 0; w < warp; ++w) before += sm.warp_act[w];
+        if (act) sm.act[before] = (int16_t)tid;
+        if (tid == 0) sm.n_active = sm.warp_act[0] + sm.warp_act[1] + sm.warp_act[2] + sm.warp_act[3];
+    }
     if (tid < P) {
         const int e = sm.idx[tid];
         int rank = 0;
@@ -109,298 +134,444 @@ __device__ __forceinline__ void build_index(const DecodeArgs& a, DecodeIndex& sm
     __syncthreads();
 }
 
-// ------------------------------------------------------------------------------ gate/up + SiLU*mul
-// Work unit: gpc consecutive 16-row groups of one active expert's gate and up matrices over the whole
-// reduction length d_model (gpc > 1 when d_model is short, so that a unit still moves tens of KB).
-// The 8 warps of a CTA split the unit's k-chunks; their partial tiles are added in warp order.
-__global__ void __launch_bounds__(kDfThreadsA, 3)
-decode_gateup_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int gpc) {
+// How a phase's units are dealt to the grid's warps: every warp gets ONE contiguous range of k-chunks.
+//   few units (fewer than 8 per CTA): ks adjacent warps of a CTA share one unit and cut its k-chunks
+//     into ks contiguous parts; warp group wg of CTA b takes unit b + gridDim * wg, so that consecutive
+//     units land in different CTAs and every busy warp has the same amount of work (more than half of
+//     the warps are busy, which is enough requests in flight to keep HBM busy);
+//   many units: CTA b takes the contiguous units [U b / G, U (b + 1) / G) and its 16 warps cut that
+//     unit-major chunk list into 16 equal contiguous ranges (CTAs differ by at most one unit in 8).
+// A range that starts inside a unit yields a "head" partial tile (left in shared memory), one that
+// starts a unit but does not finish it a "tail" (kept in registers): after the phase's streaming the
+// warp that holds a unit's tail adds the heads of the following warps in warp order.
+struct WarpWork {
+    int u0, kc0, n;       // first unit, first chunk inside it, number of chunks
+};
+__device__ __forceinline__ WarpWork deal_units(int n_units, int KC, int warp) {
+    const int G = (int)gridDim.x, b = (int)blockIdx.x;
+    WarpWork w;
+    if (n_units < 8 * G) {
+        int ks = 1;
+        while (ks < kDfWarps && ks * 2 <= KC && (long long)n_units * ks * 2 <= (long long)G * kDfWarps) ks *= 2;   // every warp of a group gets a chunk
+        const int u = b + G * (warp / ks), s = warp % ks;
+        const int c0 = KC * s / ks, c1 = KC * (s + 1) / ks;
+        w.u0 = u;
+        w.kc0 = c0;
+        w.n = u < n_units ? c1 - c0 : 0;
+    } else {
+        const int ub = (int)((long long)n_units * b / G), ue = (int)((long long)n_units * (b + 1) / G);
+        const long long n = (long long)(ue - ub) * KC;
+        const long long q0 = n * warp / kDfWarps, q1 = n * (warp + 1) / kDfWarps;
+        w.u0 = ub + (int)(q0 / KC);
+        w.kc0 = (int)(q0 % KC);
+        w.n = (int)(q1 - q0);
+    }
+    return w;
+}
+
+// A unit's address arithmetic.  PHASE 0: unit = hidden units 16j..16j+15 of expert act[ai]: 16 gate rows and the
+// 16 matching up rows, 2 KB each, contiguous in the packed tiles (the up tile follows the gate tile); activations are
+// token rows of x.  PHASE 1: unit = output columns 32j..32j+31: 32 consecutive rows of a down-matrix tile (4 KB
+// contiguous); activations are the segment's rows of h.  A chunk (64 reduction elements) of a unit is 4 KB of
+// weights: one stage.
+template <int PHASE>
+struct Unit {
+    static constexpr uint32_t kStride = PHASE == 0 ? 2u * kTileBytes : (uint32_t)kTileBytes;    // bytes between chunks
+    // first chunk's weights of unit u (the tile rows of chunk kc are + kc * kStride)
+    static __device__ __forceinline__ const uint8_t* weights(const DecodeArgs& a, const SlotTable& tab, const DecodeIndex& sm,
+                                                             int u, int upe, int KC) {
+        const int ai = u / upe, j = u - ai * upe;
+        const uint8_t* slot = a.slot_region + (size_t)tab.slot[sm.act[ai]] * a.slot_bytes;
+        if (PHASE == 0) return slot + (size_t)(j >> 3) * KC * kStride + (size_t)((j & 7) << 4) * 128u;
+        return slot + (size_t)2 * a.d * a.f * 2 + (size_t)(j >> 2) * KC * kStride + (size_t)((j & 3) << 5) * 128u;
+    }
+    // this lane's activation row (MMA column g = the segment's g-th row) at reduction element 8 t; nullptr beyond the segment
+    static __device__ __forceinline__ const uint16_t* acts(const DecodeArgs& a, const DecodeIndex& sm, int u, int upe, int g, int t) {
+        const int e = sm.act[u / upe];
+        if (g >= sm.counts[e]) return nullptr;
+        if (PHASE == 0) {
+            const int token = e < a.E ? sm.perm[sm.offsets[e] + g] / a.k : g;
+            return a.x + (size_t)token * a.d + t * 8;
+        }
+        return a.h + (size_t)(sm.offsets[e] + g) * a.f + t * 8;
+    }
+};
+
+// phase_mask: 1 = phase A, 2 = phase B, 3 = both in this launch with the grid barrier in between.
+__global__ void __launch_bounds__(kDfThreads, 1)
+decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phase_mask) {
+    extern __shared__ __align__(16) uint8_t ring_raw[];
     __shared__ DecodeIndex sm;
-    __shared__ float red[kDfWarpsA][2][kDfRows][kDfMaxTokens];
+    __shared__ float red[kDfWarps][8][32];
+    __shared__ int head_unit[kDfWarps];
+    __shared__ __align__(8) uint64_t stage_bar[kDfWarps][kDfStages];
+    __shared__ int barrier_ok, abort_flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    pdl_wait();                       // logits and x may come from the kernel before
-    pdl_launch_dependents();
-    build_index(a, sm);
+    const int g = lane >> 2, t = lane & 3;            // MMA fragment coordinates
     const int P = a.T * a.k, ES = a.E + a.S;
-    if (blockIdx.x == 0) {            // the index outputs of the step, for the caller and for inspection
-        for (int p = tid; p < P; p += kDfThreadsA) {
+    const uint32_t ring = (smem_u32(ring_raw) + 127u & ~127u) + (uint32_t)(warp * kDfStages) * kDfStageBytes;
+    const uint32_t bars = smem_u32(&stage_bar[warp][0]);
+    if (tid == 0) {
+        abort_flag = 0;
+        barrier_ok = 1;
+        for (int i = 0; i < kDfWarps * kDfStages; ++i) mbar_init(smem_u32(&stage_bar[0][0]) + 8u * i, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // A launch that starts with phase A may run ahead of the kernel that produces logits and x.  A
+    // phase-B-only launch follows the phase-A launch, which passed this very wait before it let
+    // dependents start: logits and x are final, weights are never written by a kernel, so everything
+    // up to the wait for h further down may overlap the phase-A launch.
+    if (phase_mask & 1) {
+        pdl_wait();
+        pdl_launch_dependents();
+    }
+    unsigned long long barrier_target = 0;
+    if (phase_mask == 3 && tid == 0) {                // before this CTA arrives, the counter cannot pass the next multiple of G
+        unsigned long long c;
+        asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(c) : "l"(a.sync) : "memory");
+        barrier_target = (c / gridDim.x + 1ull) * gridDim.x;
+    }
+    build_index(a, tab, sm);
+    const int n_active = sm.n_active;
+    if (blockIdx.x == 0 && (phase_mask & 1)) {        // the index outputs of the step, for the caller and for inspection
+        for (int p = tid; p < P; p += kDfThreads) {
             a.topk_idx[p] = sm.idx[p];
             a.topk_w[p] = sm.w[p];
             a.perm[p] = sm.perm[p];
             a.inv_perm[p] = sm.inv[p];
         }
-        for (int e = tid; e < ES; e += kDfThreadsA) a.counts[e] = sm.counts[e];
-        for (int e = tid; e <= ES; e += kDfThreadsA) a.offsets[e] = sm.offsets[e];
+        for (int e = tid; e < ES; e += kDfThreads) a.counts[e] = sm.counts[e];
+        for (int e = tid; e <= ES; e += kDfThreads) a.offsets[e] = sm.offsets[e];
+        if (tid == 0 && sm.absent) atomicExch(a.status, SAEM_ERR_NOT_RESIDENT);
     }
+    // byte offsets of this lane's two 16-byte pieces (k positions 8t.. and 32 + 8t.. of the chunk) in a tile row whose
+    // index is g modulo 8
+    const uint32_t piece0 = (uint32_t)((t ^ g) << 4), piece1 = (uint32_t)(((4 + t) ^ g) << 4);
 
-    const int KC = a.d / kTileK;
-    const int units_per_expert = a.f / kDfRows / gpc;
-    const int total_units = sm.n_active * units_per_expert;
-    const int wpg = kDfWarpsA / gpc;              // warps per row group
-    const int grp = warp % gpc, kslice = warp / gpc;
-    const int g = lane >> 2, t = lane & 3;        // MMA fragment coordinates
-    for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x) {
-        const int ai = unit / units_per_expert, cb = unit - ai * units_per_expert;
-        const int e = sm.act[ai];
-        const int slot = tab.slot[e];
-        if (slot < 0) {                            // routed to an expert that has no slot: rows left untouched
-            if (cb == 0 && tid == 0) atomicExch(a.status, SAEM_ERR_NOT_RESIDENT);
-            continue;
-        }
-        const int row0 = sm.offsets[e], m = sm.counts[e];
-        const int rg = cb * gpc + grp;
-        const int rb = rg >> 3, r_in = (rg & 7) * kDfRows;
-        const uint8_t* wbase = a.slot_region + (size_t)slot * a.slot_bytes + (size_t)rb * KC * (2 * kTileBytes);
-        // byte offset of this lane's 16-byte chunk (k positions 4 b + t) in tile rows r_in + g and r_in + g + 8
-        const uint32_t off_lo0 = (uint32_t)(r_in + g) * 128u + (uint32_t)((t ^ g) << 4);
-        const uint32_t off_lo1 = (uint32_t)(r_in + g) * 128u + (uint32_t)(((4 + t) ^ g) << 4);
-        const uint32_t off_hi0 = off_lo0 + 8u * 128u, off_hi1 = off_lo1 + 8u * 128u;
-        const bool x_valid = g < m;
-        // MMA column g is the segment's g-th row: the token of pair perm[row0 + g], or token g of a shared expert
-        const int token = !x_valid ? 0 : (e < a.E ? sm.perm[row0 + g] / a.k : g);
-        const uint16_t* xrow = a.x + (size_t)token * a.d + t * 8;
-
-        float cg[4] = {0.f, 0.f, 0.f, 0.f}, cu[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int kc = kslice; kc < KC; kc += wpg) {
-            const uint8_t* tile = wbase + (size_t)kc * (2 * kTileBytes);
-            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            const uint4 wl0 = *reinterpret_cast<const uint4*>(tile + off_lo0);
-            const uint4 wl1 = *reinterpret_cast<const uint4*>(tile + off_lo1);
-            const uint4 wh0 = *reinterpret_cast<const uint4*>(tile + off_hi0);
-            const uint4 wh1 = *reinterpret_cast<const uint4*>(tile + off_hi1);
-            const uint4 ul0 = *reinterpret_cast<const uint4*>(tile + kTileBytes + off_lo0);
-            const uint4 ul1 = *reinterpret_cast<const uint4*>(tile + kTileBytes + off_lo1);
-            const uint4 uh0 = *reinterpret_cast<const uint4*>(tile + kTileBytes + off_hi0);
-            const uint4 uh1 = *reinterpret_cast<const uint4*>(tile + kTileBytes + off_hi1);
-            const uint4 x0 = x_valid ? *reinterpret_cast<const uint4*>(xrow + (size_t)kc * kTileK) : z;
-            const uint4 x1 = x_valid ? *reinterpret_cast<const uint4*>(xrow + (size_t)kc * kTileK + 32) : z;
-            mma_16816(cg, wl0.x, wh0.x, wl0.y, wh0.y, x0.x, x0.y);
-            mma_16816(cg, wl0.z, wh0.z, wl0.w, wh0.w, x0.z, x0.w);
-            mma_16816(cu, ul0.x, uh0.x, ul0.y, uh0.y, x0.x, x0.y);
-            mma_16816(cu, ul0.z, uh0.z, ul0.w, uh0.w, x0.z, x0.w);
-            mma_16816(cg, wl1.x, wh1.x, wl1.y, wh1.y, x1.x, x1.y);
-            mma_16816(cg, wl1.z, wh1.z, wl1.w, wh1.w, x1.z, x1.w);
-            mma_16816(cu, ul1.x, uh1.x, ul1.y, uh1.y, x1.x, x1.y);
-            mma_16816(cu, ul1.z, uh1.z, ul1.w, uh1.w, x1.z, x1.w);
-        }
-        // accumulator fragment: c0,c1 -> (row g, tokens 2t, 2t+1); c2,c3 -> (row g + 8, same tokens)
-        red[warp][0][g][2 * t] = cg[0];
-        red[warp][0][g][2 * t + 1] = cg[1];
-        red[warp][0][g + 8][2 * t] = cg[2];
-        red[warp][0][g + 8][2 * t + 1] = cg[3];
-        red[warp][1][g][2 * t] = cu[0];
-        red[warp][1][g][2 * t + 1] = cu[1];
-        red[warp][1][g + 8][2 * t] = cu[2];
-        red[warp][1][g + 8][2 * t + 1] = cu[3];
-        __syncthreads();
-        // red[w] is the partial tile of warp w = kslice * gpc + group; a group's slices are added in order
-        for (int o = tid; o < gpc * kDfRows * kDfMaxTokens; o += kDfThreadsA) {
-            const int gq = o >> 7, n = (o >> 4) & 7, r = o & 15;
-            if (n < m) {
-                float sg = 0.f, su = 0.f;
-                for (int ks = 0; ks < wpg; ++ks) {
-                    sg += red[ks * gpc + gq][0][r][n];
-                    su += red[ks * gpc + gq][1][r][n];
-                }
-                const float hv = sg / (1.f + expf(-sg)) * su;
-                const size_t col = (size_t)(cb * gpc + gq) * kDfRows + r;
-                reinterpret_cast<__nv_bfloat16*>(a.h)[(size_t)(row0 + n) * a.f + col] = __float2bfloat16_rn(hv);
-            }
-        }
-        __syncthreads();
-    }
-}
-
-// ------------------------------------------------------------------------------- down + combine
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-
-constexpr int kDfStageBytes = 6 * 32 * 16;       // per warp and stage: 4 weight pieces + 2 activation pieces per lane
-
-// One CTA per 16 output columns (16 rows of every expert's down matrix), W warps, D stages per warp.
-// With fewer active experts than warps, wpe warps share an expert and split its k-chunks (their
-// partial tiles are added in warp order); otherwise every warp walks its own experts a, a + W, ...
-// over the whole reduction length d_ff and no partial tiles exist.
-template <int W, int D>
-__global__ void __launch_bounds__(W * 32, W <= 8 ? 2 : 1)
-decode_down_combine_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab) {
-    extern __shared__ __align__(16) uint8_t ring_raw[];
-    __shared__ DecodeIndex sm;
-    __shared__ float y_s[kDfMaxRows][kDfRows];
-    __shared__ float red[W][kDfRows][kDfMaxTokens];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // The kernel before this one in the stream (the gate/up kernel) waited for ITS predecessors
-    // before it let this kernel start, so the step's inputs (logits, x) are final here and the
-    // expert weights are never written by a kernel: everything up to the wait below may run while
-    // the gate/up kernel is still streaming.
-    for (int o = tid; o < kDfMaxRows * kDfRows; o += W * 32) (&y_s[0][0])[o] = 0.f;
-    for (int o = tid; o < W * kDfRows * kDfMaxTokens; o += W * 32) (&red[0][0][0])[o] = 0.f;   // a warp may have no chunk
-    build_index(a, sm);
-
-    const int KC = a.f / kTileK;
-    const int n_active = sm.n_active;
-    int wpe = 1;
-    while (wpe * 2 * n_active <= W) wpe *= 2;
-    const int a_step = W / wpe, kslice = warp % wpe;
-    const int rg = blockIdx.x, rb = rg >> 3, r_in = (rg & 7) * kDfRows;
-    const int g = lane >> 2, t = lane & 3;
-    const uint32_t off_lo0 = (uint32_t)(r_in + g) * 128u + (uint32_t)((t ^ g) << 4);
-    const uint32_t off_lo1 = (uint32_t)(r_in + g) * 128u + (uint32_t)(((4 + t) ^ g) << 4);
-    const uint32_t off_hi0 = off_lo0 + 8u * 128u, off_hi1 = off_lo1 + 8u * 128u;
-    const size_t down_region = (size_t)2 * a.d * a.f * 2 + (size_t)rb * KC * kTileBytes;
-    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_raw) + (uint32_t)(warp * D) * kDfStageBytes + (uint32_t)lane * 16u;
-
-    // A cursor over this warp's chunk sequence: experts ai = warp / wpe, + a_step, ...; chunks kslice, + wpe, ...
-    // Experts without a slot are skipped (their rows contribute zero and the status word is set).
-    struct Cursor { int ai, kc; };
-    auto settle = [&](Cursor& c) {               // move to the next expert that has work for this warp
-        while (c.ai < n_active && (c.kc >= KC || tab.slot[sm.act[c.ai]] < 0)) { c.ai += a_step; c.kc = kslice; }
-    };
-    auto advance = [&](Cursor& c) { c.kc += wpe; settle(c); };
-    Cursor pw = {warp / wpe, kslice};            // next chunk whose weights are to be requested
-    settle(pw);
-    Cursor ph = pw, cc = pw;                     // ... whose activations are to be requested; next chunk to consume
-
-    auto issue_w = [&](const Cursor& c, int stage) {
-        const uint8_t* tile = a.slot_region + (size_t)tab.slot[sm.act[c.ai]] * a.slot_bytes + down_region +
-                              (size_t)c.kc * kTileBytes;
-        const uint32_t dst = ring + (uint32_t)stage * kDfStageBytes;
-        cp_async16(dst, tile + off_lo0, 16);
-        cp_async16(dst + 512, tile + off_lo1, 16);
-        cp_async16(dst + 1024, tile + off_hi0, 16);
-        cp_async16(dst + 1536, tile + off_hi1, 16);
-    };
-    auto issue_h = [&](const Cursor& c, int stage) {
-        const int e = sm.act[c.ai];
-        const bool valid = g < sm.counts[e];
-        const uint16_t* hrow = a.h + (size_t)(sm.offsets[e] + (valid ? g : 0)) * a.f + (size_t)c.kc * kTileK + t * 8;
-        const uint32_t dst = ring + (uint32_t)stage * kDfStageBytes;
-        cp_async16(dst + 2048, hrow, valid ? 16u : 0u);          // lanes beyond the segment's rows: zero fill
-        cp_async16(dst + 2560, hrow + 32, valid ? 16u : 0u);
-    };
-
-    // weights of the first D chunks go out before the dependency wait
-#pragma unroll
-    for (int s = 0; s < D; ++s) {
-        if (pw.ai < n_active) { issue_w(pw, s); advance(pw); }
-        cp_async_commit();
-    }
-    pdl_wait();                                  // h is complete from here on
-    pdl_launch_dependents();
-#pragma unroll
-    for (int s = 0; s < D; ++s) {
-        if (ph.ai < n_active) { issue_h(ph, s); advance(ph); }
-        cp_async_commit();
-    }
-
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    int stage = 0;
-    auto flush = [&](int ai) {                   // this warp's tile of expert ai is complete
+    // A warp has the complete tiles of a unit: two MMA row sets s = 0, 1, four accumulators each.  Accumulator
+    // fragment: c0, c1 -> (row g, tokens 2t, 2t + 1); c2, c3 -> (row g + 8, same tokens).
+    auto finish_a = [&](int u, const float* acc) {    // set s: rows g = gate rows 8s + g, rows g + 8 = the matching up rows
+        const int upe = a.f / 16;
+        const int ai = u / upe, j = u - ai * upe;
         const int e = sm.act[ai], row0 = sm.offsets[e], m = sm.counts[e];
-        if (wpe == 1) {
-            if (2 * t < m) { y_s[row0 + 2 * t][g] = acc[0]; y_s[row0 + 2 * t][g + 8] = acc[2]; }
-            if (2 * t + 1 < m) { y_s[row0 + 2 * t + 1][g] = acc[1]; y_s[row0 + 2 * t + 1][g + 8] = acc[3]; }
-        } else {
-            red[warp][g][2 * t] = acc[0];
-            red[warp][g][2 * t + 1] = acc[1];
-            red[warp][g + 8][2 * t] = acc[2];
-            red[warp][g + 8][2 * t + 1] = acc[3];
+        __nv_bfloat16* hb = reinterpret_cast<__nv_bfloat16*>(a.h);
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            const float* c = acc + 4 * s;
+            const int col = j * 16 + 8 * s + g;
+            if (2 * t < m) hb[(size_t)(row0 + 2 * t) * a.f + col] = __float2bfloat16_rn(c[0] / (1.f + expf(-c[0])) * c[2]);
+            if (2 * t + 1 < m) hb[(size_t)(row0 + 2 * t + 1) * a.f + col] = __float2bfloat16_rn(c[1] / (1.f + expf(-c[1])) * c[3]);
         }
-        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
     };
-    while (cc.ai < n_active) {
-        cp_async_wait<D - 1>();                  // the oldest outstanding stage has landed (own bytes only)
-        const uint32_t src = ring + (uint32_t)stage * kDfStageBytes;
-        const uint4 wl0 = ld_shared_v4(src), wl1 = ld_shared_v4(src + 512);
-        const uint4 wh0 = ld_shared_v4(src + 1024), wh1 = ld_shared_v4(src + 1536);
-        const uint4 x0 = ld_shared_v4(src + 2048), x1 = ld_shared_v4(src + 2560);
-        mma_16816(acc, wl0.x, wh0.x, wl0.y, wh0.y, x0.x, x0.y);
-        mma_16816(acc, wl0.z, wh0.z, wl0.w, wh0.w, x0.z, x0.w);
-        mma_16816(acc, wl1.x, wh1.x, wl1.y, wh1.y, x1.x, x1.y);
-        mma_16816(acc, wl1.z, wh1.z, wl1.w, wh1.w, x1.z, x1.w);
-        const int ai_done = cc.ai;
-        advance(cc);
-        if (cc.ai != ai_done) flush(ai_done);
-        // refill the stage just consumed (the MMAs above have read it: they issued before this point)
-        if (pw.ai < n_active) { issue_w(pw, stage); issue_h(pw, stage); advance(pw); }
-        cp_async_commit();
-        if (++stage == D) stage = 0;
-    }
-    cp_async_wait<0>();
-    __syncthreads();
-    if (wpe > 1) {                               // add the k-slices of every expert in warp order
-        for (int o = tid; o < n_active * kDfRows * kDfMaxTokens; o += W * 32) {
-            const int ai = o >> 7, n = (o >> 4) & 7, r = o & 15;
-            const int e = sm.act[ai];
-            if (n < sm.counts[e] && tab.slot[e] >= 0) {
-                float s = 0.f;
-                for (int ks = 0; ks < wpe; ++ks) s += red[ai * wpe + ks][r][n];
-                y_s[sm.offsets[e] + n][r] = s;
+    auto finish_b = [&](int u, const float* acc) {    // store y, take a ticket for the 32 columns, merge them if last
+        const int upe = a.d / 32;
+        const int ai = u / upe, j = u - ai * upe;
+        const int e = sm.act[ai], row0 = sm.offsets[e], m = sm.counts[e];
+        float* y = a.y_packed;
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {                  // set s: rows 16 s + g and 16 s + g + 8 of the unit
+            const float* c = acc + 4 * s;
+            const int col = j * 32 + 16 * s + g;
+            if (2 * t < m) {
+                y[(size_t)(row0 + 2 * t) * a.d + col] = c[0];
+                y[(size_t)(row0 + 2 * t) * a.d + col + 8] = c[2];
+            }
+            if (2 * t + 1 < m) {
+                y[(size_t)(row0 + 2 * t + 1) * a.d + col] = c[1];
+                y[(size_t)(row0 + 2 * t + 1) * a.d + col + 8] = c[3];
+            }
+        }
+        __threadfence();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) {
+            int* ticket = a.sync + 64 + j;
+            last = atomicAdd(ticket, 1) == n_active - 1;
+            if (last) *ticket = 0;                     // every contributor has arrived: ready for the next step
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (!last) return;
+        __threadfence();
+        for (int o = lane; o < a.T * 32; o += 32) {
+            const int tok = o >> 5, c = o & 31;
+            float s = 0.f;
+            for (int jj = 0; jj < a.k; ++jj) {         // slot order, fused multiply-adds: the combine kernel's arithmetic
+                if (tab.slot[sm.idx[tok * a.k + jj]] < 0) continue;
+                s = fmaf(sm.w[tok * a.k + jj], __ldcg(y + (size_t)sm.inv[tok * a.k + jj] * a.d + j * 32 + c), s);
+            }
+            for (int sh = 0; sh < a.S; ++sh)
+                if (tab.slot[a.E + sh] >= 0) s += __ldcg(y + (size_t)(P + sh * a.T + tok) * a.d + j * 32 + c);
+            const size_t at = (size_t)tok * a.d + j * 32 + c;
+            if (a.out_bf16) reinterpret_cast<__nv_bfloat16*>(a.out)[at] = __float2bfloat16_rn(s);
+            else reinterpret_cast<float*>(a.out)[at] = s;
+        }
+    };
+
+    // The streaming loop of one phase over this warp's chunk range ww.  Lane 0 keeps kDfStages bulk copies of 4 KB
+    // in flight (request for chunk i + kDfStages goes out when chunk i has been consumed); every lane loads its own
+    // activation pieces of the NEXT chunk from L2 into registers while the current chunk's weights are awaited.
+    // `requested` chunks have been requested by the caller already.  Complete tiles are delivered through `finish`,
+    // partial ones parked.  Returns false if a wait ran out.
+    uint32_t parity = 0;                               // bit s: the phase of stage s's barrier to wait for next
+    auto stream = [&](auto unit_tag, const WarpWork& ww, int KC, int upe, auto& finish, int requested) -> bool {
+        using U = decltype(unit_tag);
+        // ---- producer state (lane 0 issues) ----
+        int pu = ww.u0, pkc = ww.kc0, pleft = ww.n;
+        const uint8_t* wp = nullptr;
+        if (pleft > 0) wp = U::weights(a, tab, sm, pu, upe, KC) + (size_t)pkc * U::kStride;
+        auto request = [&](int stage) {               // the next chunk's 4 KB into `stage`
+            if (lane == 0) {
+                const uint32_t dst = ring + (uint32_t)stage * kDfStageBytes, bar = bars + 8u * stage;
+                mbar_expect_tx(bar, 4096u);
+                if (U::kStride == 2u * kTileBytes) {   // gate rows, then the up rows of the tile behind
+                    bulk_g2s(dst, wp, 2048, bar);
+                    bulk_g2s(dst + 2048, wp + kTileBytes, 2048, bar);
+                } else {
+                    bulk_g2s(dst, wp, 4096, bar);
+                }
+            }
+            wp += U::kStride;
+            --pleft;
+            if (++pkc == KC && pleft > 0) {
+                ++pu;
+                pkc = 0;
+                wp = U::weights(a, tab, sm, pu, upe, KC);
+            }
+        };
+        // `requested` chunks are in flight already: move the producer past them, then fill the remaining stages
+        for (int s = 0; s < kDfStages; ++s) {
+            if (pleft <= 0) break;
+            if (s < requested) {
+                wp += U::kStride;
+                --pleft;
+                if (++pkc == KC && pleft > 0) { ++pu; pkc = 0; wp = U::weights(a, tab, sm, pu, upe, KC); }
+            } else {
+                request(s);
+            }
+        }
+        // ---- consumer state ----
+        float acc[8], tail[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = tail[i] = 0.f;
+        int tail_unit = -1;
+        int u = ww.u0, kc_begin = ww.kc0, left = ww.n;
+        int in_unit = KC - kc_begin < left ? KC - kc_begin : left;     // chunks of this range inside the current unit
+        int run = in_unit;
+        int stage = 0;
+        bool ok = true;
+        const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+        const uint16_t* xq = nullptr;                  // this lane's activation row at the chunk to be fetched next
+        uint4 xa = zero4, xb = zero4;                  // activation pieces of the current chunk
+        if (left > 0) {
+            xq = U::acts(a, sm, u, upe, g, t);
+            if (xq) {
+                xq += (size_t)kc_begin * kTileK;
+                xa = ld_act(xq);
+                xb = ld_act(xq + 32);
+                xq += kTileK;
+            }
+        }
+        // this lane's weight pieces inside a stage: rows g (+ 8 per set) of the first 2 KB, the matching rows 2 KB further
+        // (up rows in phase A; rows + 16 ... in phase B the second set is 2 KB further and the + 8 rows 1 KB further)
+        const uint32_t w_lo = ring + (uint32_t)g * 128u;
+        constexpr uint32_t kSetStep = U::kStride == 2u * kTileBytes ? 1024u : 2048u;     // bytes from set 0's rows g to set 1's
+        constexpr uint32_t kHiStep = U::kStride == 2u * kTileBytes ? 2048u : 1024u;      // bytes from rows g to the set's rows g + 8
+        while (left > 0) {
+            // activation pieces of the next chunk (it may belong to the next unit of this range)
+            uint4 na = zero4, nb = zero4;
+            if (left > 1) {
+                if (run == 1) xq = U::acts(a, sm, u + 1, upe, g, t);
+                if (xq) {
+                    na = ld_act(xq);
+                    nb = ld_act(xq + 32);
+                    xq += kTileK;
+                }
+            }
+            ok = mbar_wait(bars + 8u * stage, (parity >> stage) & 1u, &abort_flag, a.status, kDfBarrierLimitNs);
+            if (!ok) break;
+            parity ^= 1u << stage;
+            const uint32_t base = w_lo + (uint32_t)stage * kDfStageBytes;
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                const uint32_t lo = base + (uint32_t)s * kSetStep, hi = lo + kHiStep;
+                const uint4 w00 = ld_shared_v4(lo + piece0), w01 = ld_shared_v4(lo + piece1);
+                const uint4 w10 = ld_shared_v4(hi + piece0), w11 = ld_shared_v4(hi + piece1);
+                mma_16816(acc + 4 * s, w00.x, w10.x, w00.y, w10.y, xa.x, xa.y);
+                mma_16816(acc + 4 * s, w00.z, w10.z, w00.w, w10.w, xa.z, xa.w);
+                mma_16816(acc + 4 * s, w01.x, w11.x, w01.y, w11.y, xb.x, xb.y);
+                mma_16816(acc + 4 * s, w01.z, w11.z, w01.w, w11.w, xb.z, xb.w);
+            }
+            __syncwarp();                              // every lane has read the stage (its MMAs issued) before it is refilled
+            if (pleft > 0) request(stage);
+            if (++stage == kDfStages) stage = 0;
+            xa = na;
+            xb = nb;
+            --left;
+            if (--run == 0) {                          // this range's share of unit u is complete
+                if (kc_begin > 0) {                    // started inside the unit: a head partial
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) red[warp][i][lane] = acc[i];
+                    if (lane == 0) head_unit[warp] = u;
+                } else if (in_unit < KC) {             // started the unit but does not finish it: the tail
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) tail[i] = acc[i];
+                    tail_unit = u;
+                } else {
+                    finish(u, acc);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+                ++u;
+                kc_begin = 0;
+                in_unit = KC < left ? KC : left;
+                run = in_unit;
             }
         }
         __syncthreads();
-    }
-    if (blockIdx.x == 0 && tid < n_active && tab.slot[sm.act[tid]] < 0) atomicExch(a.status, SAEM_ERR_NOT_RESIDENT);
-    // merge: slot order j = 0..k-1 with fused multiply-adds, then the shared experts with weight 1
-    const int P = a.T * a.k;
-    for (int o = tid; o < a.T * kDfRows; o += W * 32) {
-        const int tok = o >> 4, c = o & 15;
-        float s = 0.f;
-        for (int j = 0; j < a.k; ++j) s = fmaf(sm.w[tok * a.k + j], y_s[sm.inv[tok * a.k + j]][c], s);
-        for (int sh = 0; sh < a.S; ++sh) s += y_s[P + sh * a.T + tok][c];
-        const size_t at = (size_t)tok * a.d + (size_t)rg * kDfRows + c;
-        if (a.out_bf16) reinterpret_cast<__nv_bfloat16*>(a.out)[at] = __float2bfloat16_rn(s);
-        else reinterpret_cast<float*>(a.out)[at] = s;
-    }
-}
+        if (ok && tail_unit >= 0 && !abort_flag) {     // add the following warps' heads in warp order
+            for (int w2 = warp + 1; w2 < kDfWarps && head_unit[w2] == tail_unit; ++w2)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) tail[i] += red[w2][i][lane];
+            finish(tail_unit, tail);
+        }
+        return ok;
+    };
 
-// Row groups per unit of the gate/up kernel: enough that a unit moves about 64 KB of weights, a power
-// of two that divides both the warp count and the number of row groups.
-static int groups_per_unit(int rows, int K) {
-    const int n_groups = rows / kDfRows;
-    const long long bytes_per_group = (long long)kDfRows * K * 2 * 2;
-    int gpc = 1;
-    while (gpc < kDfWarpsA && bytes_per_group * gpc < 64 * 1024 && n_groups % (gpc * 2) == 0) gpc *= 2;
-    return gpc;
+    // ================================ phase A: gate/up + SiLU*mul ================================
+    if (phase_mask & 1) {
+        const int KC = a.d / kTileK, upe = a.f / 16;
+        const WarpWork ww = deal_units(n_active * upe, KC, warp);
+        if (lane == 0) head_unit[warp] = -1;
+        stream(Unit<0>(), ww, KC, upe, finish_a, 0);
+    }
+
+    // ================================ phase B: down + merge ================================
+    if (phase_mask & 2) {
+        const int KC = a.f / kTileK, upe = a.d / 32;
+        const WarpWork ww = deal_units(n_active * upe, KC, warp);
+        if (phase_mask == 3) __syncthreads();          // phase A's readers of head_unit are done
+        if (lane == 0) head_unit[warp] = -1;
+        // weights of the first stages go out before this warp meets the grid (or waits for the phase-A launch)
+        int requested = 0;
+        {
+            int pu = ww.u0, pkc = ww.kc0;
+            for (; requested < kDfStages && requested < ww.n; ++requested) {
+                if (lane == 0) {
+                    const uint32_t dst = ring + (uint32_t)requested * kDfStageBytes, bar = bars + 8u * requested;
+                    mbar_expect_tx(bar, 4096u);
+                    bulk_g2s(dst, Unit<1>::weights(a, tab, sm, pu, upe, KC) + (size_t)pkc * Unit<1>::kStride, 4096, bar);
+                }
+                if (++pkc == KC) { ++pu; pkc = 0; }
+            }
+        }
+        bool ok = true;
+        if (phase_mask == 3) {
+            // Grid barrier: every h store of phase A is visible device-wide before anyone reads h.  The CTA's
+            // stores are ordered before thread 0's release by the CTA barrier (release / acquire are cumulative).
+            // The arrival counter only ever grows: G arrivals per launch, so this launch is complete when the
+            // counter reaches the next multiple of G above what thread 0 saw when the kernel started.
+            __syncthreads();
+            if (tid == 0) {
+                int good = abort_flag ? 0 : 1;
+                unsigned long long* counter = reinterpret_cast<unsigned long long*>(a.sync);
+                asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(counter) : "memory");
+                unsigned long long t0 = 0;
+                for (uint32_t i = 0;; ++i) {
+                    unsigned long long c;
+                    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(c) : "l"(counter) : "memory");
+                    if (c >= barrier_target) break;
+                    if ((i & 255u) == 255u) {
+                        const unsigned long long now = globaltimer_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > kDfBarrierLimitNs) { good = 0; atomicExch(a.status, SAEM_ERR_TIMEOUT); break; }
+                    }
+                }
+                barrier_ok = good;
+            }
+            __syncthreads();
+            ok = barrier_ok != 0;
+        } else {
+            pdl_wait();                                // h is complete from here on
+            pdl_launch_dependents();
+        }
+        if (ok) stream(Unit<1>(), ww, KC, upe, finish_b, requested);
+    }
+    // Copies still in flight (a wait that ran out, a barrier that was not met) must land before the CTA's shared
+    // memory goes away.
+    if (abort_flag || (phase_mask == 3 && !barrier_ok)) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) {}
+    }
 }
 
 bool decode_fused_supported(int T, int k) { return T >= 1 && T <= kDfMaxTokens && k <= kDfMaxK; }
 
+// mode per device: 0 not decided, 1 cooperative + programmatic serialization, 2 cooperative, 3 two launches
+static int g_mode[64];
+
+static cudaError_t launch_step(const DecodeArgs& a, const SlotTable& tab, int grid, cudaStream_t st, int phase_mask,
+                               bool cooperative, bool pdl) {
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (cooperative) {
+        attr[n].id = cudaLaunchAttributeCooperative;
+        attr[n].val.cooperative = 1;
+        ++n;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kDfThreads);
+    cfg.dynamicSmemBytes = kDfRingBytes;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, decode_step_kernel, a, tab, phase_mask);
+}
+
 cudaError_t launch_decode_fused(const DecodeArgs& a, const SlotTable& tab, int n_sm, cudaStream_t st, int* n_launch) {
-    constexpr int kBigSmem = 16 * 4 * kDfStageBytes, kSmallSmem = 8 * 3 * kDfStageBytes;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     static bool attr_done[64];
     if (first_call_on_device(attr_done)) {
-        cudaError_t e = cudaFuncSetAttribute(decode_down_combine_kernel<16, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBigSmem);
+        e = cudaFuncSetAttribute(decode_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDfRingBytes);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(decode_down_combine_kernel<8, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmallSmem);
-        if (e != cudaSuccess) return e;
+        int coop = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) coop = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_step_kernel, kDfThreads, kDfRingBytes) != cudaSuccess)
+            per_sm = 0;
+        g_mode[dev] = (coop && per_sm >= 1) ? 0 : 3;
     }
-    const int gpc = groups_per_unit(a.f, a.d);
-    const int units_per_expert = a.f / kDfRows / gpc;
-    const long long bound_active = (long long)a.T * a.k + a.S < a.E + a.S ? (long long)a.T * a.k + a.S : a.E + a.S;
-    long long grid_a = bound_active * units_per_expert;
-    if (grid_a > 3LL * n_sm) grid_a = 3LL * n_sm;
-    if (grid_a < 1) grid_a = 1;
-    cudaError_t e = launch_pdl(decode_gateup_kernel, dim3((unsigned)grid_a), dim3(kDfThreadsA), 0, st, a, tab, gpc);
+    const int grid = n_sm;                     // one CTA per SM
+    if (g_mode[dev] == 0) {                    // first step on this device: find out what the driver accepts
+        e = launch_step(a, tab, grid, st, 3, true, true);
+        if (e == cudaSuccess) { g_mode[dev] = 1; *n_launch = 1; return e; }
+        (void)cudaGetLastError();
+        e = launch_step(a, tab, grid, st, 3, true, false);
+        if (e == cudaSuccess) { g_mode[dev] = 2; *n_launch = 1; return e; }
+        (void)cudaGetLastError();
+        g_mode[dev] = 3;
+    }
+    if (g_mode[dev] == 1 || g_mode[dev] == 2) {
+        *n_launch = 1;
+        return launch_step(a, tab, grid, st, 3, true, g_mode[dev] == 1);
+    }
+    e = launch_step(a, tab, grid, st, 1, false, true);
     if (e != cudaSuccess) return e;
-    const int grid_b = a.d / kDfRows;
-    // one CTA per SM with 16 warps and four stages each when the column groups fit one wave; otherwise
-    // two smaller CTAs per SM
-    if (grid_b <= n_sm)
-        e = launch_pdl(decode_down_combine_kernel<16, 4>, dim3((unsigned)grid_b), dim3(16 * 32), (size_t)kBigSmem, st, a, tab);
-    else
-        e = launch_pdl(decode_down_combine_kernel<8, 3>, dim3((unsigned)grid_b), dim3(8 * 32), (size_t)kSmallSmem, st, a, tab);
     *n_launch = 2;
-    return e;
+    return launch_step(a, tab, grid, st, 2, false, true);
+}
+
+int decode_fused_mode() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    return g_mode[dev];
 }
 
 }  // namespace saem

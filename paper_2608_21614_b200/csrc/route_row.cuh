@@ -46,11 +46,12 @@ __device__ __forceinline__ void route_row(const float* __restrict__ row, int E, 
         unsigned long long best = key[0];
 #pragma unroll
         for (int i = 1; i < kPerLane; ++i) best = key[i] > best ? key[i] : best;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-            best = other > best ? other : best;
-        }
+        // warp-wide maximum of the 64-bit key in two 32-bit reductions: the largest value word, then
+        // the largest ~id (the lowest expert id) among the lanes that hold that value
+        const uint32_t hi = (uint32_t)(best >> 32);
+        const uint32_t hi_max = __reduce_max_sync(0xffffffffu, hi);
+        const uint32_t lo_max = __reduce_max_sync(0xffffffffu, hi == hi_max ? (uint32_t)best : 0u);
+        best = ((unsigned long long)hi_max << 32) | lo_max;
         int e = (int)(~(uint32_t)best);
         float v = key_value((uint32_t)(best >> 32));
         if (j == 0) {

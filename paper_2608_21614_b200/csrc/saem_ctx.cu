@@ -24,7 +24,7 @@ int validate_config(const saem_config* c) {
     if (c->temp_slots < 0 || c->temp_slots > 4096) return SAEM_ERR_SHAPE;
     if ((long long)c->n_layers * c->slots_per_layer + c->temp_slots < 1) return SAEM_ERR_SHAPE;
     if (c->out_dtype != SAEM_OUT_F32 && c->out_dtype != SAEM_OUT_BF16) return SAEM_ERR_INVALID_ARG;
-    if (c->ffn_path < SAEM_FFN_AUTO || c->ffn_path > SAEM_FFN_TENSOR_PAIRS) return SAEM_ERR_INVALID_ARG;
+    if (c->ffn_path < SAEM_FFN_AUTO || c->ffn_path > SAEM_FFN_DECODE_FUSED) return SAEM_ERR_INVALID_ARG;
     // repack keeps a [pairs/32][E] table of 16-bit counters in shared memory
     long long chunks = ((long long)c->max_tokens * c->top_k + 31) / 32;
     if (chunks * c->n_experts * 2 > 160 * 1024) return SAEM_ERR_UNSUPPORTED;
@@ -48,6 +48,7 @@ WorkspaceLayout workspace_layout(const saem_config& c) {
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, A); return o; };
     L.status = take(256);
     L.counters = take(sizeof(int) * 2 * kMaxCtas);
+    L.decode_sync = take(sizeof(int) * kDecodeSyncInts);
     L.h = take(R * f * 2);
     {   // split-K partial tiles of the streaming kernels: token tiles of at most 64 rows, two slots per CTA
         size_t small_tile = (size_t)2 * (nt < 64 ? nt : 64) * kTileRows;
@@ -175,7 +176,7 @@ int saem_create(const saem_config* cfg, void* slot_region, size_t slot_region_by
     for (int i = 0; ok && i < cfg->n_layers; ++i)
         ok = cudaEventCreateWithFlags(&c->read_ev[i], cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaHostAlloc((void**)&c->pinned_status, sizeof(int), cudaHostAllocDefault) == cudaSuccess;
-    // the status word and the split-K arrival counters start at zero; nothing else needs clearing
+    // the status word, the arrival counters and the decode step's barrier / tickets start at zero; nothing else needs clearing
     ok = ok && cudaMemsetAsync(c->ws + lay.status, 0, lay.h - lay.status, 0) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(0) == cudaSuccess;
     if (ok && cfg->ffn_path != SAEM_FFN_SCALAR) ok = ffn_tensor_init() == cudaSuccess;
@@ -373,7 +374,7 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     const int seg_bound = max_rows < g.max_tokens ? max_rows : g.max_tokens;     // a token picks an expert once
     if (g.ffn_path == SAEM_FFN_SCALAR) {
         CUDA_TRY(launch_ffn_scalar(a, tab, st, &nl));
-    } else if (g.ffn_path == SAEM_FFN_AUTO && seg_bound <= 8) {
+    } else if ((g.ffn_path == SAEM_FFN_AUTO || g.ffn_path == SAEM_FFN_DECODE_FUSED) && seg_bound <= 8) {
         CUDA_TRY(launch_ffn_gemv(a, tab, st, &nl));
     } else {
         CUDA_TRY(launch_ffn_tensor(a, tab, st, &nl));
@@ -422,9 +423,10 @@ int saem_moe_step(saem_ctx* c, saem_ctx* sh, int layer, const float* logits, con
     int32_t* inv = (int32_t*)(w + L.inv_perm);
     float* y = (float*)(w + L.y_packed);
     float* shy = (float*)(w + L.shared_y);
-    if (!sh && g.ffn_path == SAEM_FFN_AUTO && decode_fused_supported(T, g.top_k)) {
-        // The smallest decode batches: two launches for the whole step (gate + repack indices + gate/up,
-        // then down + merge); x_packed and y_packed are not produced.
+    if (!sh && decode_fused_supported(T, g.top_k) &&
+        (g.ffn_path == SAEM_FFN_DECODE_FUSED || (g.ffn_path == SAEM_FFN_AUTO && T <= kDecodeFusedAutoTokens))) {
+        // The smallest decode batches: one launch for the whole step (gate + repack indices + gate/up,
+        // grid barrier, down + merge); x_packed is not produced.
         if (layer < 0 || layer >= g.n_layers) return SAEM_ERR_INVALID_ARG;
         if (misaligned(x) || misaligned(out)) return SAEM_ERR_ALIGNMENT;
         cudaStream_t st = (cudaStream_t)stream;
@@ -435,6 +437,8 @@ int saem_moe_step(saem_ctx* c, saem_ctx* sh, int layer, const float* logits, con
         a.T = T; a.E = g.n_experts; a.S = g.n_shared; a.k = g.top_k; a.d = g.d_model; a.f = g.d_ff; a.renorm = g.renorm;
         a.slot_region = c->slot_region; a.slot_bytes = c->slot_bytes;
         a.h = (uint16_t*)(w + L.h);
+        a.y_packed = y;
+        a.sync = (int*)(w + L.decode_sync);
         a.out = out; a.out_bf16 = g.out_dtype == SAEM_OUT_BF16;
         a.topk_idx = idx; a.topk_w = tw; a.counts = (int32_t*)(w + L.counts); a.offsets = offsets;
         a.perm = (int32_t*)(w + L.perm); a.inv_perm = inv;
@@ -587,7 +591,7 @@ int saem_last_device_status(saem_ctx* c, int* code) {
     CUDA_TRY(cudaMemset(c->ws + c->lay.status, 0, sizeof(int)));
     // a CTA that gave up a bounded wait skipped its arrival on a split item's counter: start the next
     // launch from clean counters (nothing is in flight after the synchronisation above)
-    if (*code == SAEM_ERR_TIMEOUT) CUDA_TRY(cudaMemset(c->ws + c->lay.counters, 0, sizeof(int) * 2 * kMaxCtas));
+    if (*code == SAEM_ERR_TIMEOUT) CUDA_TRY(cudaMemset(c->ws + c->lay.counters, 0, c->lay.h - c->lay.counters));
     return SAEM_OK;
 }
 

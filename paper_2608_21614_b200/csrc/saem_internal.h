@@ -27,6 +27,7 @@ struct SlotTable {
 struct WorkspaceLayout {
     size_t status;        // int32 status word (+ padding)
     size_t counters;      // int32[2 * kMaxCtas] split-K arrival counters (gate/up, down)
+    size_t decode_sync;   // int32[kDecodeSyncInts] grid barrier and column-group tickets of the one-launch decode step
     size_t h;             // bf16 [max_rows, d_ff]
     size_t partials;      // fp32 [CTAs][2][2][n_tile][128]: 2 CTAs/SM for n_tile <= 64, else 1 CTA/SM
     size_t logits, x, topk_idx, topk_w, counts, offsets, perm, inv_perm, x_packed, y_packed, shared_y, out;
@@ -126,8 +127,9 @@ cudaError_t launch_ffn_scalar(const FfnArgs& a, const SlotTable& tab, cudaStream
 cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
 // Segments of at most 8 rows (decode batches 1..8): row-split matrix-vector kernels.
 cudaError_t launch_ffn_gemv(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
-// The whole step for batches of at most 8 tokens (top_k at most 8) in two launches: gate + repack
-// indices + gate/up projection, then down projection + merge (decode_fused.cu).
+// The whole step for batches of at most 8 tokens (top_k at most 8) in one launch (two where a
+// cooperative launch is not available): gate + repack indices + gate/up projection, grid barrier,
+// down projection + merge (decode_fused.cu).
 struct DecodeArgs {
     const float* logits;        // [T, E]
     const uint16_t* x;          // [T, d]
@@ -135,6 +137,8 @@ struct DecodeArgs {
     const uint8_t* slot_region;
     size_t slot_bytes;
     uint16_t* h;                // [T * (k + S), f] bf16 workspace
+    float* y_packed;            // [T * (k + S), d] fp32 workspace
+    int* sync;                  // [0..1] 64-bit count of barrier arrivals (only grows), [64 + j] ticket of output columns 32j..32j+31
     void* out;                  // [T, d]
     int out_bf16;
     int32_t* topk_idx;          // index outputs of the step, written by one CTA
@@ -146,7 +150,11 @@ struct DecodeArgs {
     int* status;
 };
 bool decode_fused_supported(int T, int k);
+// SAEM_FFN_AUTO takes the one-launch step up to this many tokens (measured: faster than the five-launch
+// step at 1..4 tokens on every layer shape tried, slower at 8)
+constexpr int kDecodeFusedAutoTokens = 4;
 cudaError_t launch_decode_fused(const DecodeArgs& a, const SlotTable& tab, int n_sm, cudaStream_t st, int* n_launch);
+constexpr int kDecodeSyncInts = 64 + 1024;   // d_model <= 16384: at most 1024 groups of 16 columns
 // One-time per process: resolves the driver entry point for tensor-map encoding and opts the
 // kernels into large dynamic shared memory.  Returns cudaSuccess or the failing error.
 cudaError_t ffn_tensor_init();

@@ -83,6 +83,30 @@ def run_stepwise_and_compare(layer, li, oracle, ref=None):
     return ref, stats
 
 
+def run_single_call_and_compare(layer, li, oracle, ref=None):
+    """The whole step through saem_moe_step (for at most 8 tokens: the two-launch decode path) against
+    the oracle: the index outputs left in the workspace bit-exact, the layer output within tolerance."""
+    c = li.cfg
+    T, k, E = c.tokens, c.top_k, c.n_experts
+    P, ES = T * k, c.n_experts + layer.S
+    if ref is None:
+        ref = oracle.moe_step(li.logits, li.x, k, li.gate, li.up, li.down, shared=li.shared)
+    out = torch.full((T, c.d_model), float("nan"), dtype=torch.float32, device=layer.device)
+    layer.step_fused_call(dev(li.logits), dev(li.x), T, out)
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    ctx = layer.ctx
+    assert np.array_equal(host(ctx.step_tensor(0, (T, k), torch.int32)), ref["topk_idx"]), "topk_idx"
+    assert np.abs(host(ctx.step_tensor(1, (T, k), torch.float32)).astype(np.float64) - ref["topk_w"]).max() <= W_TOL
+    counts, offsets = host(ctx.step_tensor(2, (ES,), torch.int32)), host(ctx.step_tensor(3, (ES + 1,), torch.int32))
+    assert np.array_equal(counts[:E], ref["counts"]) and np.array_equal(offsets[:E + 1], ref["offsets"])
+    if layer.S:
+        assert np.all(counts[E:] == T) and np.array_equal(offsets[E:], P + T * np.arange(layer.S + 1))
+    assert np.array_equal(host(ctx.step_tensor(4, (P,), torch.int32)), ref["perm"]), "perm"
+    assert np.array_equal(host(ctx.step_tensor(5, (P,), torch.int32)), ref["inv_perm"]), "inv_perm"
+    return ref, assert_close(host(out), ref["out"], "out of the single-call step")
+
+
 # ------------------------------------------------------------------ partially resident stacks
 def run_stack(trace, weights, L, E, k, d, f, C, temp, batch, steps, keep, policy="stage", eap=None):
     from paper_2608_21614_b200.stack import StackRunner

@@ -34,6 +34,20 @@ def test_fine_grained_decode_full(oracle, name, T, routing):
     layer.close()
 
 
+@pytest.mark.parametrize("name,T", [("c4", 1), ("c4", 4), ("c4", 8), ("qwen3", 1), ("qwen3", 4), ("qwen3", 8),
+                                    ("ernie", 1), ("ernie", 8), ("c5", 1), ("c5", 4), ("c5", 8)])
+def test_single_launch_decode_step_full_shapes(oracle, name, T):
+    """The two-launch decode step (saem_moe_step, at most 8 tokens) on the layer shapes of the
+    benchmark configurations and of the paper's two models."""
+    import gpu_util as g
+    li = gen.layer_inputs(gen.layer_config(name, tokens=T), n_distinct_experts=4)
+    layer = g.make_layer(li, 4)                     # SAEM_FFN_DECODE_FUSED: the one-launch form up to 8 tokens
+    n0 = layer.launches()
+    g.run_single_call_and_compare(layer, li, oracle)
+    assert layer.launches() - n0 in (1, 2)      # one cooperative launch, or two where that is not available
+    layer.close()
+
+
 PAIRS = 3       # SAEM_FFN_TENSOR_PAIRS: the CTA-pair form of the tiled kernels wherever the shape allows
 
 

@@ -9,7 +9,7 @@ from paper_2608_21614_b200 import inputs as gen
 
 pytestmark = pytest.mark.gpu
 
-AUTO, SCALAR, TENSOR, PAIRS = 0, 1, 2, 3
+AUTO, SCALAR, TENSOR, PAIRS, FUSED = 0, 1, 2, 3, 4
 
 
 @pytest.fixture(scope="module")
@@ -38,7 +38,7 @@ def test_c1_every_call(oracle, path):
 
 
 @pytest.mark.parametrize("T,E,k,d,f,fs", [(1, 1, 1, 128, 128, 0), (1, 60, 4, 256, 384, 256), (1, 60, 4, 256, 384, 384),
-                                          (8, 8, 8, 128, 256, 0), (5, 128, 8, 256, 128, 128), (8, 8, 2, 512, 1024, 0),
+                                          (8, 8, 8, 128, 256, 0), (5, 120, 8, 256, 128, 128), (8, 8, 2, 512, 1024, 0),
                                           (3, 16, 2, 2048, 1408, 2816)])
 def test_tiny_batches_matrix_vector_path(oracle, T, E, k, d, f, fs):
     """Batches of at most 8 tokens take the row-split matrix-vector kernels (ffn_path AUTO)."""
@@ -51,6 +51,65 @@ def test_tiny_batches_matrix_vector_path(oracle, T, E, k, d, f, fs):
     layer.step(g.dev(li.logits), g.dev(li.x), T)
     torch.cuda.synchronize()
     assert torch.equal(y1, layer.y_packed)                 # deterministic
+    layer.close()
+
+
+@pytest.mark.parametrize("T,E,k,d,f,fs", [(1, 1, 1, 128, 128, 0), (1, 60, 4, 256, 384, 384), (8, 8, 8, 128, 256, 0),
+                                          (5, 120, 8, 256, 128, 128), (8, 8, 2, 512, 1024, 0), (7, 33, 5, 384, 640, 0),
+                                          (3, 16, 2, 2048, 1408, 2816), (8, 12, 1, 256, 128, 2048), (2, 8, 2, 2432, 256, 0)])
+def test_single_launch_decode_step(oracle, T, E, k, d, f, fs):
+    """saem_moe_step for at most 8 tokens (top-k at most 8): gate, repack indices, gate/up, down
+    projection and merge in one launch.  Index outputs bit-exact, output within tolerance, run to
+    run bit-identical, and (bf16 hidden activations, fp32 sums on both sides) close to the four
+    separate calls."""
+    g = _g()
+    cfg = gen.LayerConfig("t", d, f, E, k, T, fs, "zipf", 1.1, seed=200 + T + E)
+    li = gen.layer_inputs(cfg, n_distinct_experts=min(E, 6))
+    layer = g.make_layer(li, FUSED)
+    assert layer.shared is None
+    n0 = layer.launches()
+    ref, _ = g.run_single_call_and_compare(layer, li, oracle)
+    assert layer.launches() - n0 in (1, 2)      # one cooperative launch, or two where that is not available
+    logits, x = g.dev(li.logits), g.dev(li.x)
+    o1 = torch.empty((T, d), dtype=torch.float32, device="cuda:0")
+    o2 = torch.empty_like(o1)
+    layer.step_fused_call(logits, x, T, o1)
+    layer.step_fused_call(logits, x, T, o2)
+    four = layer.step(logits, x, T)
+    torch.cuda.synchronize()
+    assert torch.equal(o1, o2)
+    assert float((o1 - four).abs().max()) <= 2e-3
+    layer.close()
+
+
+def test_single_launch_decode_step_bf16_out_and_absent_expert(oracle, B):
+    """bf16 output of the two-launch step, and a routed expert without a slot: the status word says
+    NOT_RESIDENT and the expert contributes nothing (the other experts' terms are still merged)."""
+    g = _g()
+    cfg = gen.LayerConfig("t", 256, 384, 6, 2, 4, 0, "normal", seed=31)
+    li = gen.layer_inputs(cfg)
+    from paper_2608_21614_b200.layer import MoELayer
+    layer = g.make_layer(li, FUSED, out_dtype=B.SAEM_OUT_BF16)
+    out = torch.zeros((4, 256), dtype=torch.uint16, device="cuda:0")
+    layer.step_fused_call(g.dev(li.logits), g.dev(li.x), 4, out)
+    torch.cuda.synchronize()
+    ref = oracle.moe_step(li.logits, li.x, 2, li.gate, li.up, li.down)
+    g.assert_close(gen.bf16_bits_to_f32(g.host(out)), ref["out"], "bf16 out")
+    layer.close()
+    missing = int(ref["topk_idx"][0, 0])
+    layer = MoELayer(256, 384, 6, 2, 4)
+    for e in range(6):
+        if e != missing:
+            layer.load_expert(0, e, e, li.gate[e], li.up[e], li.down[e])
+    o = torch.zeros((4, 256), dtype=torch.float32, device="cuda:0")
+    layer.step_fused_call(g.dev(li.logits), g.dev(li.x), 4, o)
+    torch.cuda.synchronize()
+    assert layer.device_status() == B.SAEM_ERR_NOT_RESIDENT
+    zero = [np.zeros_like(m) for m in (li.gate[missing], li.up[missing], li.down[missing])]
+    gate, up, down = list(li.gate), list(li.up), list(li.down)
+    gate[missing], up[missing], down[missing] = zero
+    ref2 = oracle.moe_step(li.logits, li.x, 2, gate, up, down)
+    g.assert_close(g.host(o), ref2["out"], "absent expert contributes zero")
     layer.close()
 
 
