@@ -60,6 +60,7 @@ typedef enum saem_status {
 
 enum { SAEM_MAX_EXPERTS = 128 };         /* routed experts per layer */
 enum { SAEM_TEMP = -2 };                 /* slot argument of saem_cache_load: take a temporary slot */
+enum { SAEM_HOST_MAPPED = -3 };          /* slot reported by saem_cache_query for an expert bound by saem_cache_map_host */
 enum { SAEM_OUT_F32 = 0, SAEM_OUT_BF16 = 1 };
 enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TENSOR_PAIRS = 3, SAEM_FFN_DECODE_FUSED = 4 };
 
@@ -77,9 +78,8 @@ enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TEN
  * (tcgen05 cta_group::2: 256 tokens x 512 weight rows per pair of SMs), which AUTO and TENSOR take
  * for long reductions and many rows (d_model >= 4096, d_model % 256 == 0, at least 1536 packed
  * rows in the call); SAEM_FFN_TENSOR_PAIRS is SAEM_FFN_TENSOR with the pair form whenever
- * d_model % 256 == 0 (for tests and measurements).  SAEM_FFN_DECODE_FUSED is SAEM_FFN_AUTO, except that
- * saem_moe_step takes its one-launch form (see there) for every batch it supports (up to 8 tokens, top_k
- * up to 8) instead of up to 4 tokens.
+ * d_model % 256 == 0 (for tests and measurements).  SAEM_FFN_DECODE_FUSED is SAEM_FFN_AUTO with the
+ * one-launch form of saem_moe_step (see there) stated explicitly; SAEM_FFN_TENSOR never takes that form.
  * n_shared (0..16, n_experts + n_shared <= SAEM_MAX_EXPERTS): always-on shared experts of the same
  * width d_ff that run INSIDE the layer's grouped launch.  They are experts n_experts ..
  * n_experts + n_shared - 1 of every layer for the cache calls (outside the routed cache-ratio
@@ -212,7 +212,7 @@ int saem_combine(saem_ctx* ctx, const float* y_packed, const int32_t* inv_perm, 
  * holds an always-on shared expert whose width is not a multiple of d_ff (otherwise use
  * config.n_shared and pass NULL).
  * logits[T, E] fp32, x[T, d] bf16, out[T, d] (all dev).
- * Smallest decode batches (ffn_path AUTO: T <= 4; top_k <= 8; no shared_ctx): the whole step runs as ONE
+ * Smallest decode batches (ffn_path AUTO or DECODE_FUSED: T <= 8; top_k <= 8; no shared_ctx): the whole step runs as ONE
  * kernel launch -- gate, repack indices and gate/up projection, a grid-wide barrier, down projection and
  * merge -- launched cooperatively (two launches where the device refuses that).  topk_idx, topk_w, counts,
  * offsets, perm, inv_perm, h and y_packed are still left in the workspace; x_packed is not produced.  A
@@ -252,6 +252,19 @@ void* saem_step_buffer(saem_ctx* ctx, int which);
 int saem_cache_load(saem_ctx* ctx, int layer, int expert, int slot, const void* pinned_packed_expert,
                     void* copy_stream);
 int saem_cache_evict(saem_ctx* ctx, int layer, int expert);
+/*
+ * Binds an expert that has no slot to a packed expert in MAPPED PINNED HOST memory (cudaHostAlloc /
+ * cudaHostRegister; saem_slot_bytes, 16-byte aligned), to be read in place over the host link by the
+ * matrix-vector kernels of saem_expert_ffn (calls whose segments have at most 8 rows, ffn_path AUTO): the
+ * GPU-side analogue of executing a missed expert where its weights are (Sec. IV-D in-situ execution; the
+ * Sec. VI ablation's on-demand transfer through a temporary slot is the other way).  No copy, no slot, no
+ * event: the memory must stay valid and unchanged until the FFNs that use it have finished.  Every other
+ * kernel treats such an expert as absent, and saem_moe_step takes its five-launch form for a layer that
+ * has one.  At most 8 host-mapped experts per FFN call (UNSUPPORTED beyond).  saem_cache_evict removes
+ * the binding; a slot loaded later takes precedence.  Errors: INVALID_ARG (has a slot; not mapped pinned
+ * memory), ALIGNMENT.
+ */
+int saem_cache_map_host(saem_ctx* ctx, int layer, int expert, const void* pinned_packed_expert);
 int saem_cache_query(saem_ctx* ctx, int layer, int expert, int* slot, int* ready);
 int saem_cache_wait(saem_ctx* ctx, int layer, int expert, void* consumer_stream);
 

@@ -20,6 +20,7 @@ SAEM_ERR_INVALID_ARG, SAEM_ERR_SHAPE, SAEM_ERR_ALIGNMENT, SAEM_ERR_WORKSPACE = 1
 SAEM_ERR_NOT_RESIDENT, SAEM_ERR_SLOT_BUSY, SAEM_ERR_TIMEOUT, SAEM_ERR_CUDA, SAEM_ERR_UNSUPPORTED = 5, 6, 7, 8, 9
 SAEM_MAX_EXPERTS = 128
 SAEM_TEMP = -2
+SAEM_HOST_MAPPED = -3
 SAEM_OUT_F32, SAEM_OUT_BF16 = 0, 1
 SAEM_FFN_AUTO, SAEM_FFN_SCALAR, SAEM_FFN_TENSOR, SAEM_FFN_TENSOR_PAIRS, SAEM_FFN_DECODE_FUSED = 0, 1, 2, 3, 4
 
@@ -62,6 +63,7 @@ def _load() -> C.CDLL:
         "saem_step_buffer": (vp, [vp, i32]),
         "saem_cache_load": (i32, [vp, i32, i32, i32, vp, vp]),
         "saem_cache_evict": (i32, [vp, i32, i32]),
+        "saem_cache_map_host": (i32, [vp, i32, i32, vp]),
         "saem_cache_query": (i32, [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]),
         "saem_cache_wait": (i32, [vp, i32, i32, vp]),
         "saem_last_device_status": (i32, [vp, C.POINTER(i32)]),
@@ -79,7 +81,7 @@ def _load() -> C.CDLL:
 _lib = _load()
 EXPORTS = ("saem_version saem_status_string saem_slot_bytes saem_slot_region_bytes saem_workspace_bytes "
            "saem_create saem_destroy saem_pack_expert_host saem_route saem_route_fused saem_repack saem_expert_ffn saem_combine "
-           "saem_moe_step saem_moe_step_host saem_step_buffer saem_cache_load saem_cache_evict saem_cache_query "
+           "saem_moe_step saem_moe_step_host saem_step_buffer saem_cache_load saem_cache_evict saem_cache_map_host saem_cache_query "
            "saem_cache_wait saem_last_device_status saem_launch_count saem_expert_ffn_static saem_selftest_bounded_wait").split()
 
 
@@ -234,6 +236,13 @@ def saem_cache_evict(ctx, layer, expert, check=True) -> int:
     code = _lib.saem_cache_evict(ctx, layer, expert)
     if check:
         _check(code, "saem_cache_evict")
+    return code
+
+
+def saem_cache_map_host(ctx, layer, expert, pinned_packed_expert, check=True) -> int:
+    code = _lib.saem_cache_map_host(ctx, layer, expert, _ptr(pinned_packed_expert))
+    if check:
+        _check(code, "saem_cache_map_host")
     return code
 
 

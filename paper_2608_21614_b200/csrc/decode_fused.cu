@@ -139,13 +139,16 @@ __device__ __forceinline__ void build_index(const DecodeArgs& a, const SlotTable
 //     into ks contiguous parts; warp group wg of CTA b takes unit b + gridDim * wg, so that consecutive
 //     units land in different CTAs and every busy warp has the same amount of work (more than half of
 //     the warps are busy, which is enough requests in flight to keep HBM busy);
-//   many units: CTA b takes the contiguous units [U b / G, U (b + 1) / G) and its 16 warps cut that
-//     unit-major chunk list into 16 equal contiguous ranges (CTAs differ by at most one unit in 8).
+//   many units: CTA b takes the units b, b + G, b + 2 G, ... (every CTA gets a share of every expert, so
+//     an expert that streams faster or slower than the others -- its weights partly in L2, more rows --
+//     does not unbalance the grid) and its 16 warps cut that unit-major chunk list into 16 equal
+//     contiguous ranges (CTAs differ by at most one unit in 8).
 // A range that starts inside a unit yields a "head" partial tile (left in shared memory), one that
 // starts a unit but does not finish it a "tail" (kept in registers): after the phase's streaming the
 // warp that holds a unit's tail adds the heads of the following warps in warp order.
 struct WarpWork {
     int u0, kc0, n;       // first unit, first chunk inside it, number of chunks
+    int ustep;            // distance between consecutive units of this warp's range
 };
 __device__ __forceinline__ WarpWork deal_units(int n_units, int KC, int warp) {
     const int G = (int)gridDim.x, b = (int)blockIdx.x;
@@ -158,13 +161,15 @@ __device__ __forceinline__ WarpWork deal_units(int n_units, int KC, int warp) {
         w.u0 = u;
         w.kc0 = c0;
         w.n = u < n_units ? c1 - c0 : 0;
+        w.ustep = 1;
     } else {
-        const int ub = (int)((long long)n_units * b / G), ue = (int)((long long)n_units * (b + 1) / G);
-        const long long n = (long long)(ue - ub) * KC;
+        const int mine = (n_units - b + G - 1) / G;    // units b, b + G, b + 2 G, ...
+        const long long n = (long long)mine * KC;
         const long long q0 = n * warp / kDfWarps, q1 = n * (warp + 1) / kDfWarps;
-        w.u0 = ub + (int)(q0 / KC);
+        w.u0 = b + G * (int)(q0 / KC);
         w.kc0 = (int)(q0 % KC);
         w.n = (int)(q1 - q0);
+        w.ustep = G;
     }
     return w;
 }
@@ -333,7 +338,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             wp += U::kStride;
             --pleft;
             if (++pkc == KC && pleft > 0) {
-                ++pu;
+                pu += ww.ustep;
                 pkc = 0;
                 wp = U::weights(a, tab, sm, pu, upe, KC);
             }
@@ -344,7 +349,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             if (s < requested) {
                 wp += U::kStride;
                 --pleft;
-                if (++pkc == KC && pleft > 0) { ++pu; pkc = 0; wp = U::weights(a, tab, sm, pu, upe, KC); }
+                if (++pkc == KC && pleft > 0) { pu += ww.ustep; pkc = 0; wp = U::weights(a, tab, sm, pu, upe, KC); }
             } else {
                 request(s);
             }
@@ -380,7 +385,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             // activation pieces of the next chunk (it may belong to the next unit of this range)
             uint4 na = zero4, nb = zero4;
             if (left > 1) {
-                if (run == 1) xq = U::acts(a, sm, u + 1, upe, g, t);
+                if (run == 1) xq = U::acts(a, sm, u + ww.ustep, upe, g, t);
                 if (xq) {
                     na = ld_act(xq);
                     nb = ld_act(xq + 32);
@@ -421,7 +426,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
                 }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-                ++u;
+                u += ww.ustep;
                 kc_begin = 0;
                 in_unit = KC < left ? KC : left;
                 run = in_unit;
@@ -461,7 +466,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
                     mbar_expect_tx(bar, 4096u);
                     bulk_g2s(dst, Unit<1>::weights(a, tab, sm, pu, upe, KC) + (size_t)pkc * Unit<1>::kStride, 4096, bar);
                 }
-                if (++pkc == KC) { ++pu; pkc = 0; }
+                if (++pkc == KC) { pu += ww.ustep; pkc = 0; }
             }
         }
         bool ok = true;

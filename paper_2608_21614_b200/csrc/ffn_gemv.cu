@@ -56,7 +56,7 @@ ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, int gpc) {
             if (r1 > a.max_rows) r1 = a.max_rows;
             rows = r1 > r0 ? r1 - r0 : 0;
             if (!tab.in_subset[e]) rows = 0;
-            if (rows > 0 && tab.slot[e] < 0) {
+            if (rows > 0 && tab.slot[e] == -1) {
                 if (blockIdx.x == 0 && blockIdx.y == 0) atomicExch(a.status, SAEM_ERR_NOT_RESIDENT);
                 rows = 0;
             }
@@ -90,7 +90,9 @@ ffn_gemv_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, int gpc) {
     const int kslice = warp / gpc;
     const int rb = rg >> 3, r_in = (rg & 7) * kGvRows;
     const int g = lane >> 2, t = lane & 3;     // MMA fragment coordinates
-    const uint8_t* slot = a.slot_region + (size_t)tab.slot[e] * a.slot_bytes;
+    // an HBM slot, or a packed expert in mapped pinned host memory read in place over the host link
+    const int si = tab.slot[e];
+    const uint8_t* slot = si >= 0 ? a.slot_region + (size_t)si * a.slot_bytes : tab.host[-(si + 2)];
     const uint8_t* wbase = PHASE == 0 ? slot + (size_t)rb * KC * (2 * kTileBytes)
                                       : slot + (size_t)2 * a.d * a.f * 2 + (size_t)rb * KC * kTileBytes;
     const size_t chunk_stride = PHASE == 0 ? 2 * kTileBytes : kTileBytes;

@@ -10,7 +10,8 @@
 //
 // Small problems (pairs <= kFusedPairs): every CTA of the grid repeats the index phase in its own
 // shared memory (only CTA 0 writes the index outputs) and then copies its share of the rows, so
-// the whole repack is one launch.  Larger problems: one index CTA, then a grid-wide gather.
+// the whole repack is one launch.  Larger problems: the index phase runs on one CTA per 1024 pairs in
+// two passes (per-block histograms and ranks; offsets and scatter), then a grid-wide gather.
 #include "saem_internal.h"
 
 namespace saem {
@@ -35,12 +36,9 @@ struct RepackSmem {
 };
 static_assert(sizeof(RepackSmem) % 16 == 0, "the chunk table must start 16-byte aligned");
 
-// Shared-memory carve: [RepackSmem][chunk table uint16 n_chunks*E][rank uint8 P_padded][perm int32 P (fused only)]
-// e8 (optional, P bytes): the expert ids staged in shared memory by one sweep of coalesced loads
-// that are all in flight together (255 = invalid); without it every warp pays a global-memory
-// round trip per 32-pair chunk, which is most of the index kernel's time at prefill sizes.
+// Shared-memory carve: [RepackSmem][chunk table uint16 n_chunks*E][perm int32 P][rank uint8 P_padded]
 __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int P, int E, int S, int T, RepackSmem& sm,
-                                            uint16_t* table, uint8_t* rank, uint8_t* e8, int32_t* perm_s, bool write_global,
+                                            uint16_t* table, uint8_t* rank, int32_t* perm_s, bool write_global,
                                             int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                                             int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
                                             int* __restrict__ status) {
@@ -56,28 +54,11 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
         for (int i = tid; i < n16; i += blockDim.x) t4[i] = make_uint4(0u, 0u, 0u, 0u);
     }
     if (tid == 0) sm.bad = 0;
-    if (e8) {
-        __syncthreads();                             // sm.bad is cleared before anyone may set it
-        for (int p0 = tid; p0 < P; p0 += 4 * blockDim.x) {
-            int v[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { const int p = p0 + u * blockDim.x; v[u] = p < P ? idx[p] : 0; }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int p = p0 + u * blockDim.x;
-                if (p < P) {
-                    const bool okv = v[u] >= 0 && v[u] < E;
-                    if (!okv) sm.bad = 1;
-                    e8[p] = okv ? (uint8_t)v[u] : (uint8_t)255;
-                }
-            }
-        }
-    }
     __syncthreads();
     for (int c = warp; c < n_chunks; c += n_warps) {
         int p = c * 32 + lane;
-        int e = p >= P ? -1 : e8 ? (e8[p] == 255 ? -1 : (int)e8[p]) : idx[p];
-        if (!e8 && p < P && (e < 0 || e >= E)) { e = -1; sm.bad = 1; }
+        int e = p >= P ? -1 : idx[p];
+        if (p < P && (e < 0 || e >= E)) { e = -1; sm.bad = 1; }
         // lanes with the same expert id: one ballot per bit of the id (the index phase runs on one SM
         // and is bound by its instruction issue, so only the bits that E needs); invalid pairs are
         // masked out and never use their rank
@@ -137,7 +118,7 @@ __device__ __forceinline__ void index_phase(const int32_t* __restrict__ idx, int
         if (tid == 0 && sm.bad) atomicExch(status, SAEM_ERR_INVALID_ARG);
     }
     for (int p = tid; p < P; p += blockDim.x) {
-        int e = e8 ? (e8[p] == 255 ? -1 : (int)e8[p]) : idx[p];
+        int e = idx[p];
         if (e < 0 || e >= E) { if (write_global) inv_perm[p] = -1; continue; }
         int r = sm.offsets[e] + table[e * tstride + (p >> 5)] + rank[p];
         if (perm_s) perm_s[r] = p;
@@ -173,7 +154,7 @@ repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict_
     int32_t* perm_s = reinterpret_cast<int32_t*>(smem_raw + off);
     uint8_t* rank = smem_raw + off + (size_t)n_chunks * 32 * 4;
     for (int i = threadIdx.x; i < n_chunks * 32; i += blockDim.x) perm_s[i] = -1;
-    index_phase(idx, P, E, S, T, sm, table, rank, nullptr, perm_s, blockIdx.x == 0, counts, offsets, perm, inv_perm, status);
+    index_phase(idx, P, E, S, T, sm, table, rank, perm_s, blockIdx.x == 0, counts, offsets, perm, inv_perm, status);
     const int total = sm.offsets[E];                 // rows actually packed (pairs with a valid expert)
     // each CTA copies rows r = blockIdx.x, blockIdx.x + gridDim.x, ...; 128 threads per row
     const int sub = threadIdx.x >> 7, nsub = blockDim.x >> 7;
@@ -185,20 +166,111 @@ repack_fused_kernel(const int32_t* __restrict__ idx, const uint16_t* __restrict_
         copy_row(x + (size_t)(r % T) * d, x_packed + (size_t)(P + r) * d, d, threadIdx.x & 127, 128);
 }
 
-__global__ void __launch_bounds__(1024)
-repack_index_kernel(const int32_t* __restrict__ idx, int T, int E, int S, int k, int stage_ids,
-                    int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ perm,
-                    int32_t* __restrict__ inv_perm, int* __restrict__ status) {
-    extern __shared__ __align__(16) uint8_t smem_raw[];
+// ---- larger problems: the index phase on many CTAs ----
+// Block b owns pairs [b * kBlockPairs, (b + 1) * kBlockPairs).  Pass 1: per block and expert the number of
+// pairs (hist[b][e]) and every pair's rank among the block's pairs of the same expert (rank16[p]), both by
+// the chunk rule of the one-CTA phase (ballots inside a 32-pair chunk, a scan down the block's 32 chunks).
+// Pass 2: every block adds up the columns of hist (segment offsets = scan over the expert totals; its own
+// base per expert = offset + the blocks before it) and writes perm / inv_perm for its pairs.  Ascending
+// pair id inside a segment holds by construction: blocks in order, ranks in order.
+constexpr int kBlockPairs = 1024;
+constexpr int kBlockChunks = kBlockPairs / 32;
+
+__global__ void __launch_bounds__(kBlockPairs)
+repack_hist_kernel(const int32_t* __restrict__ idx, int P, int E, int32_t* __restrict__ hist, uint16_t* __restrict__ rank16,
+                   int* __restrict__ status) {
+    __shared__ uint16_t table[SAEM_MAX_EXPERTS][kBlockChunks + 2];      // [expert][chunk], padded against bank conflicts
+    __shared__ int bad;
     pdl_wait();
     pdl_launch_dependents();
-    const int P = T * k, n_chunks = (P + 31) >> 5;
-    RepackSmem& sm = *reinterpret_cast<RepackSmem*>(smem_raw);
-    uint16_t* table = reinterpret_cast<uint16_t*>(smem_raw + sizeof(RepackSmem));
-    uint8_t* rank = smem_raw + sizeof(RepackSmem) + (((size_t)table_stride(n_chunks) * E * 2 + 15) & ~(size_t)15);
-    uint8_t* e8 = stage_ids ? rank + (size_t)n_chunks * 32 : nullptr;
-    int32_t* perm_s = stage_ids > 1 ? reinterpret_cast<int32_t*>(rank + (size_t)n_chunks * 64) : nullptr;
-    index_phase(idx, P, E, S, T, sm, table, rank, e8, perm_s, true, counts, offsets, perm, inv_perm, status);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int id_bits = E > 1 ? 32 - __clz(E - 1) : 0;
+    for (int i = tid; i < SAEM_MAX_EXPERTS * (kBlockChunks + 2); i += kBlockPairs) (&table[0][0])[i] = 0;
+    if (tid == 0) bad = 0;
+    __syncthreads();
+    const int p = blockIdx.x * kBlockPairs + tid;
+    int e = p < P ? idx[p] : -1;
+    if (p < P && (e < 0 || e >= E)) { e = -1; bad = 1; }
+    unsigned grp = __ballot_sync(0xffffffffu, e >= 0);
+    for (int b = 0; b < id_bits; ++b) {
+        const unsigned bal = __ballot_sync(0xffffffffu, (e >> b) & 1);
+        grp &= ((e >> b) & 1) ? bal : ~bal;
+    }
+    const int r = __popc(grp & ((1u << lane) - 1u));
+    if (e >= 0 && r == 0) table[e][warp] = (uint16_t)__popc(grp);
+    __syncthreads();
+    for (int x = warp; x < E; x += kBlockChunks) {                      // exclusive scan down the 32 chunks of expert x
+        const int v = table[x][lane];
+        int inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int n = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += n;
+        }
+        table[x][lane] = (uint16_t)(inc - v);
+        if (lane == 31) hist[(size_t)blockIdx.x * E + x] = inc;
+    }
+    __syncthreads();
+    if (e >= 0) rank16[p] = (uint16_t)(table[e][warp] + r);
+    if (tid == 0 && bad) atomicExch(status, SAEM_ERR_INVALID_ARG);
+}
+
+__global__ void __launch_bounds__(kBlockPairs)
+repack_scatter_kernel(const int32_t* __restrict__ idx, int T, int E, int S, int k, const int32_t* __restrict__ hist,
+                      const uint16_t* __restrict__ rank16, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                      int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+    __shared__ int total[SAEM_MAX_EXPERTS], base[SAEM_MAX_EXPERTS], seg[SAEM_MAX_EXPERTS + 1];
+    pdl_wait();
+    pdl_launch_dependents();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int P = T * k, n_blocks = (P + kBlockPairs - 1) / kBlockPairs;
+    if (tid < E) {
+        int before = 0, all = 0;
+        for (int b = 0; b < n_blocks; ++b) {
+            const int v = hist[(size_t)b * E + tid];
+            if (b < (int)blockIdx.x) before += v;
+            all += v;
+        }
+        total[tid] = all;
+        base[tid] = before;
+    }
+    __syncthreads();
+    if (warp == 0) {                                   // exclusive scan over the expert totals
+        int carry = 0;
+        for (int b0 = 0; b0 < E; b0 += 32) {
+            const int x = b0 + lane;
+            const int v = x < E ? total[x] : 0;
+            int inc = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int n = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += n;
+            }
+            if (x < E) seg[x] = carry + inc - v;
+            carry += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (lane == 0) seg[E] = carry;
+    }
+    __syncthreads();
+    const int p = blockIdx.x * kBlockPairs + tid;
+    if (p < P) {
+        const int e = idx[p];
+        if (e < 0 || e >= E) {
+            inv_perm[p] = -1;
+        } else {
+            const int r = seg[e] + base[e] + rank16[p];
+            perm[r] = p;
+            inv_perm[p] = r;
+        }
+    }
+    // rows behind the last segment hold no pair (pairs with an invalid expert id were dropped)
+    for (int r = seg[E] + (int)blockIdx.x * kBlockPairs + tid; r < P; r += (int)gridDim.x * kBlockPairs) perm[r] = -1;
+    if (blockIdx.x == 0) {
+        for (int x = tid; x < E; x += kBlockPairs) counts[x] = total[x];
+        for (int x = tid; x <= E; x += kBlockPairs) offsets[x] = seg[x];
+        if (S > 0 && tid == 0) offsets[E] = P;         // in-layer shared experts: one segment of all T tokens each
+        for (int sh = tid; sh < S; sh += kBlockPairs) { counts[E + sh] = T; offsets[E + sh + 1] = P + (sh + 1) * T; }
+    }
 }
 
 __global__ void __launch_bounds__(256)
@@ -221,17 +293,15 @@ repack_gather_kernel(const uint16_t* __restrict__ x, const int32_t* __restrict__
 
 cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, int S, int k, int d, int32_t* counts,
                           int32_t* offsets, int32_t* perm, int32_t* inv_perm, uint16_t* x_packed, int* status,
-                          int n_sm, cudaStream_t st, int* n_launch) {
+                          int32_t* hist, uint16_t* rank16, int n_sm, cudaStream_t st, int* n_launch) {
     const int P = T * k, n_chunks = (P + 31) >> 5;
-    size_t base = sizeof(RepackSmem) + (((size_t)table_stride(n_chunks) * E * 2 + 15) & ~(size_t)15);
     static bool attr_done[64];
     if (first_call_on_device(attr_done)) {
-        cudaError_t e = cudaFuncSetAttribute(repack_index_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(repack_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(repack_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
         if (e != cudaSuccess) return e;
     }
     if (P <= kFusedPairs) {
+        size_t base = sizeof(RepackSmem) + (((size_t)table_stride(n_chunks) * E * 2 + 15) & ~(size_t)15);
         size_t smem = base + (size_t)n_chunks * 32 * 4 + (size_t)n_chunks * 32;
         int rows_per_cta = kRepackThreads / 128;
         int grid = (P + S * T + rows_per_cta - 1) / rows_per_cta;
@@ -241,14 +311,13 @@ cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, i
         return launch_pdl(repack_fused_kernel, dim3(grid), dim3(kRepackThreads), smem, st, idx, x, T, E, S, k, d,
                           counts, offsets, perm, inv_perm, x_packed, status);
     }
-    size_t smem = base + (size_t)n_chunks * 32;
-    // when they fit too: the expert ids staged in shared memory (1), and the permutation as well (2)
-    const int stage_ids = smem + (size_t)n_chunks * 32 * 5 <= 200 * 1024 ? 2 : smem + (size_t)n_chunks * 32 <= 200 * 1024 ? 1 : 0;
-    if (stage_ids) smem += (size_t)n_chunks * 32 * (stage_ids == 2 ? 5 : 1);
-    cudaError_t e = launch_pdl(repack_index_kernel, dim3(1), dim3(1024), smem, st, idx, T, E, S, k, stage_ids, counts,
-                               offsets, perm, inv_perm, status);
+    const int n_blocks = (P + kBlockPairs - 1) / kBlockPairs;
+    cudaError_t e = launch_pdl(repack_hist_kernel, dim3(n_blocks), dim3(kBlockPairs), 0, st, idx, P, E, hist, rank16, status);
     if (e != cudaSuccess) return e;
-    *n_launch = 2;
+    e = launch_pdl(repack_scatter_kernel, dim3(n_blocks), dim3(kBlockPairs), 0, st, idx, T, E, S, k, (const int32_t*)hist,
+                   (const uint16_t*)rank16, counts, offsets, perm, inv_perm);
+    if (e != cudaSuccess) return e;
+    *n_launch = 3;
     return launch_pdl(repack_gather_kernel, dim3(n_sm * 4), dim3(256), 0, st, x, perm, offsets, T, E, S, k, d, x_packed);
 }
 

@@ -25,11 +25,6 @@ int validate_config(const saem_config* c) {
     if ((long long)c->n_layers * c->slots_per_layer + c->temp_slots < 1) return SAEM_ERR_SHAPE;
     if (c->out_dtype != SAEM_OUT_F32 && c->out_dtype != SAEM_OUT_BF16) return SAEM_ERR_INVALID_ARG;
     if (c->ffn_path < SAEM_FFN_AUTO || c->ffn_path > SAEM_FFN_DECODE_FUSED) return SAEM_ERR_INVALID_ARG;
-    // repack keeps a [pairs/32][E] table of 16-bit counters in shared memory
-    long long chunks = ((long long)c->max_tokens * c->top_k + 31) / 32;
-    if (chunks * c->n_experts * 2 > 160 * 1024) return SAEM_ERR_UNSUPPORTED;
-    // ... next to a rank byte per pair (rows of the table are padded by up to three entries)
-    if ((chunks + 3) * c->n_experts * 2 + chunks * 32 + 2048 > 200 * 1024) return SAEM_ERR_UNSUPPORTED;
     return SAEM_OK;
 }
 
@@ -53,6 +48,11 @@ WorkspaceLayout workspace_layout(const saem_config& c) {
     {   // split-K partial tiles of the streaming kernels: token tiles of at most 64 rows, two slots per CTA
         size_t small_tile = (size_t)2 * (nt < 64 ? nt : 64) * kTileRows;
         L.partials = take((size_t)kMaxCtas * 2 * small_tile * sizeof(float));
+    }
+    {   // multi-CTA repack (more than 2048 pairs): at most 64 blocks of 1024 pairs
+        const bool big = P > 2048;
+        L.repack_hist = take(big ? (size_t)64 * SAEM_MAX_EXPERTS * 4 : 16);
+        L.repack_rank = take(big ? (size_t)65536 * 2 : 16);
     }
     L.logits = take(T * (size_t)c.n_experts * 4);
     L.x = take(T * d * 2);
@@ -154,6 +154,7 @@ int saem_create(const saem_config* cfg, void* slot_region, size_t slot_region_by
     size_t LE = (size_t)cfg->n_layers * c->n_total;
     c->slot_of = (int32_t*)malloc(sizeof(int32_t) * LE);
     c->temp_of = (int32_t*)malloc(sizeof(int32_t) * LE);
+    c->host_of = (const uint8_t**)calloc(LE, sizeof(const uint8_t*));
     c->slot_owner = (int32_t*)malloc(sizeof(int32_t) * n_slots);
     c->ready_ev = (cudaEvent_t*)calloc(n_slots, sizeof(cudaEvent_t));
     c->ev_pending = (uint8_t*)calloc(n_slots, 1);
@@ -198,7 +199,7 @@ void saem_destroy(saem_ctx* c) {
         for (int i = 0; i < c->cfg.n_layers; ++i)
             if (c->read_ev[i]) cudaEventDestroy(c->read_ev[i]);
     if (c->pinned_status) cudaFreeHost(c->pinned_status);
-    free(c->slot_of); free(c->temp_of); free(c->slot_owner); free(c->ready_ev); free(c->ev_pending);
+    free(c->slot_of); free(c->temp_of); free(c->host_of); free(c->slot_owner); free(c->ready_ev); free(c->ev_pending);
     free(c->ev_recorded); free(c->read_ev); free(c->read_recorded); free(c->temp_last_layer); free(c->last_stream); free(c->ffn_seen);
     delete c;
 }
@@ -275,7 +276,8 @@ int saem_repack(saem_ctx* c, const int32_t* idx, const void* x, int T, int32_t* 
     if (misaligned(x) || misaligned(x_packed)) return SAEM_ERR_ALIGNMENT;
     int nl = 0;
     CUDA_TRY(launch_repack(idx, (const uint16_t*)x, T, c->cfg.n_experts, c->cfg.n_shared, c->cfg.top_k, c->cfg.d_model, counts,
-                           offsets, perm, inv_perm, (uint16_t*)x_packed, (int*)(c->ws + c->lay.status), c->n_sm,
+                           offsets, perm, inv_perm, (uint16_t*)x_packed, (int*)(c->ws + c->lay.status),
+                           (int32_t*)(c->ws + c->lay.repack_hist), (uint16_t*)(c->ws + c->lay.repack_rank), c->n_sm,
                            (cudaStream_t)stream, &nl));
     c->launches += nl;
     return SAEM_OK;
@@ -283,22 +285,41 @@ int saem_repack(saem_ctx* c, const int32_t* idx, const void* x, int T, int32_t* 
 
 // Slot of every expert of `layer` for one FFN launch (fixed slot, else temporary binding, else -1),
 // and `st` ordered after the loads still in flight for those slots.
-static int resolve_slots(saem_ctx* c, int layer, const int32_t* subset, int n_subset, cudaStream_t st, SlotTable& tab) {
+static int resolve_slots(saem_ctx* c, int layer, const int32_t* subset, int n_subset, cudaStream_t st, SlotTable& tab,
+                         bool host_mapped_ok = false) {
     const int ES = c->n_total;
     const int32_t* so = c->slot_of + (size_t)layer * ES;
     const int32_t* to = c->temp_of + (size_t)layer * ES;
+    const uint8_t* const* ho = c->host_of + (size_t)layer * ES;
     for (int e = 0; e < SAEM_MAX_EXPERTS; ++e) { tab.slot[e] = -1; tab.in_subset[e] = 0; }
-    auto resolve = [&](int e) { return so[e] >= 0 ? so[e] : to[e]; };
+    for (int i = 0; i < kMaxHostMapped; ++i) tab.host[i] = nullptr;
+    int n_host = 0;
+    bool too_many = false;
+    // fixed slot, else temporary binding, else (where the kernels can read it) mapped host memory
+    auto resolve = [&](int e) -> int {
+        if (so[e] >= 0) return so[e];
+        if (to[e] >= 0) return to[e];
+        if (ho[e] && host_mapped_ok) {
+            if (n_host == kMaxHostMapped) { too_many = true; return -1; }
+            tab.host[n_host] = ho[e];
+            return -(2 + n_host++);
+        }
+        return -1;
+    };
     if (subset) {
         for (int i = 0; i < n_subset; ++i) {
             int e = subset[i];
             if (e < 0 || e >= ES) return SAEM_ERR_INVALID_ARG;
-            if (resolve(e) < 0) return SAEM_ERR_NOT_RESIDENT;
+            if (so[e] < 0 && to[e] < 0 && !(ho[e] && host_mapped_ok)) return SAEM_ERR_NOT_RESIDENT;
         }
-        for (int i = 0; i < n_subset; ++i) { tab.slot[subset[i]] = resolve(subset[i]); tab.in_subset[subset[i]] = 1; }
+        for (int i = 0; i < n_subset; ++i) {
+            if (!tab.in_subset[subset[i]]) tab.slot[subset[i]] = resolve(subset[i]);
+            tab.in_subset[subset[i]] = 1;
+        }
     } else {
         for (int e = 0; e < ES; ++e) { tab.slot[e] = resolve(e); tab.in_subset[e] = 1; }
     }
+    if (too_many) return SAEM_ERR_UNSUPPORTED;
     // order this stream after loads still in flight for the slots it may read
     for (int e = 0; e < ES; ++e) {
         int s = tab.slot[e];
@@ -341,9 +362,11 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     if (subset && n_subset < 0) return SAEM_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
 
+    const int seg_bound = max_rows < g.max_tokens ? max_rows : g.max_tokens;     // a token picks an expert once
+    const bool gemv_path = (g.ffn_path == SAEM_FFN_AUTO || g.ffn_path == SAEM_FFN_DECODE_FUSED) && seg_bound <= 8;
     SlotTable tab;
     {
-        int r = resolve_slots(c, layer, subset, n_subset, st, tab);
+        int r = resolve_slots(c, layer, subset, n_subset, st, tab, gemv_path);
         if (r != SAEM_OK) return r;
     }
 
@@ -371,10 +394,9 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     a.n_sm = c->n_sm;
     a.force_pairs = g.ffn_path == SAEM_FFN_TENSOR_PAIRS;
     int nl = 0;
-    const int seg_bound = max_rows < g.max_tokens ? max_rows : g.max_tokens;     // a token picks an expert once
     if (g.ffn_path == SAEM_FFN_SCALAR) {
         CUDA_TRY(launch_ffn_scalar(a, tab, st, &nl));
-    } else if ((g.ffn_path == SAEM_FFN_AUTO || g.ffn_path == SAEM_FFN_DECODE_FUSED) && seg_bound <= 8) {
+    } else if (gemv_path) {
         CUDA_TRY(launch_ffn_gemv(a, tab, st, &nl));
     } else {
         CUDA_TRY(launch_ffn_tensor(a, tab, st, &nl));
@@ -423,7 +445,10 @@ int saem_moe_step(saem_ctx* c, saem_ctx* sh, int layer, const float* logits, con
     int32_t* inv = (int32_t*)(w + L.inv_perm);
     float* y = (float*)(w + L.y_packed);
     float* shy = (float*)(w + L.shared_y);
-    if (!sh && decode_fused_supported(T, g.top_k) &&
+    bool host_mapped = false;
+    if (layer >= 0 && layer < g.n_layers)
+        for (int e = 0; e < c->n_total; ++e) host_mapped = host_mapped || c->host_of[(size_t)layer * c->n_total + e] != nullptr;
+    if (!sh && !host_mapped && decode_fused_supported(T, g.top_k) &&
         (g.ffn_path == SAEM_FFN_DECODE_FUSED || (g.ffn_path == SAEM_FFN_AUTO && T <= kDecodeFusedAutoTokens))) {
         // The smallest decode batches: one launch for the whole step (gate + repack indices + gate/up,
         // grid barrier, down + merge); x_packed is not produced.
@@ -539,10 +564,29 @@ int saem_cache_load(saem_ctx* c, int layer, int expert, int slot, const void* pi
     return SAEM_OK;
 }
 
+int saem_cache_map_host(saem_ctx* c, int layer, int expert, const void* pinned) {
+    int s = check_le(c, layer, expert);
+    if (s != SAEM_OK) return s;
+    if (!pinned || ((uintptr_t)pinned & 15)) return pinned ? SAEM_ERR_ALIGNMENT : SAEM_ERR_INVALID_ARG;
+    size_t le = (size_t)layer * c->n_total + expert;
+    if (c->slot_of[le] >= 0 || c->temp_of[le] >= 0) return SAEM_ERR_INVALID_ARG;     // it has a slot: evict first
+    void* dev = nullptr;
+    if (cudaHostGetDevicePointer(&dev, const_cast<void*>(pinned), 0) != cudaSuccess || !dev) {
+        (void)cudaGetLastError();
+        return SAEM_ERR_INVALID_ARG;                                                  // not mapped pinned memory
+    }
+    c->host_of[le] = (const uint8_t*)dev;
+    return SAEM_OK;
+}
+
 int saem_cache_evict(saem_ctx* c, int layer, int expert) {
     int s = check_le(c, layer, expert);
     if (s != SAEM_OK) return s;
     size_t le = (size_t)layer * c->n_total + expert;
+    if (c->host_of[le]) {
+        c->host_of[le] = nullptr;
+        if (c->slot_of[le] < 0 && c->temp_of[le] < 0) return SAEM_OK;
+    }
     if (c->slot_of[le] >= 0) {
         c->slot_owner[c->slot_of[le]] = -1;
         c->slot_of[le] = -1;
@@ -561,6 +605,11 @@ int saem_cache_query(saem_ctx* c, int layer, int expert, int* slot, int* ready) 
     if (s != SAEM_OK) return s;
     size_t le = (size_t)layer * c->n_total + expert;
     int gs = c->slot_of[le] >= 0 ? c->slot_of[le] : c->temp_of[le];
+    if (gs < 0 && c->host_of[le]) {                  // bound to mapped host memory: nothing to wait for
+        if (slot) *slot = SAEM_HOST_MAPPED;
+        if (ready) *ready = 1;
+        return SAEM_OK;
+    }
     if (slot) *slot = gs;
     if (ready) {
         *ready = 0;

@@ -19,9 +19,13 @@ constexpr int kMaxNTile = 256;              // widest token tile (the MMA N)
 
 // Slot index per expert for one FFN launch; travels as a kernel parameter so that the residency
 // table never needs a device mirror.  -1: the expert has no slot or is outside the subset.
+// An expert bound to mapped pinned host memory (saem_cache_map_host) has slot -(2 + i) and its weights at
+// host[i]; only the matrix-vector kernels read such experts, every other kernel sees them as absent.
+constexpr int kMaxHostMapped = 8;
 struct SlotTable {
     int32_t slot[SAEM_MAX_EXPERTS];
     uint8_t in_subset[SAEM_MAX_EXPERTS];    // 0: skip silently (not asked for)
+    const uint8_t* host[kMaxHostMapped];
 };
 
 struct WorkspaceLayout {
@@ -30,6 +34,8 @@ struct WorkspaceLayout {
     size_t decode_sync;   // int32[kDecodeSyncInts] grid barrier and column-group tickets of the one-launch decode step
     size_t h;             // bf16 [max_rows, d_ff]
     size_t partials;      // fp32 [CTAs][2][2][n_tile][128]: 2 CTAs/SM for n_tile <= 64, else 1 CTA/SM
+    size_t repack_hist;   // int32 [64][SAEM_MAX_EXPERTS] per-block histograms of the multi-CTA repack
+    size_t repack_rank;   // uint16 [65536] rank of a pair inside its block and expert
     size_t logits, x, topk_idx, topk_w, counts, offsets, perm, inv_perm, x_packed, y_packed, shared_y, out;
     size_t total;
     int n_tile_max;
@@ -97,10 +103,11 @@ cudaError_t launch_route(const float* logits, int T, int E, int k, int renorm, i
                          cudaStream_t st);
 cudaError_t launch_route_fused(const uint16_t* x, const uint16_t* w_router, int T, int E, int d, int k, int renorm,
                                float* logits_out, int32_t* idx, float* w, cudaStream_t st);
-// Returns the number of kernels launched (1 or 2) in *n_launch.
+// Returns the number of kernels launched (1 or 3) in *n_launch.  hist [ceil(P / 1024)][E] and rank16 [P]: workspace
+// of the multi-CTA index phase (more than 2048 pairs).
 cudaError_t launch_repack(const int32_t* idx, const uint16_t* x, int T, int E, int S, int k, int d, int32_t* counts,
                           int32_t* offsets, int32_t* perm, int32_t* inv_perm, uint16_t* x_packed, int* status,
-                          int n_sm, cudaStream_t st, int* n_launch);
+                          int32_t* hist, uint16_t* rank16, int n_sm, cudaStream_t st, int* n_launch);
 cudaError_t launch_combine(const float* y, const int32_t* inv_perm, const float* w, int T, int k, int S, int d,
                            const float* shared_y, void* out, int out_bf16, cudaStream_t st);
 
@@ -150,9 +157,9 @@ struct DecodeArgs {
     int* status;
 };
 bool decode_fused_supported(int T, int k);
-// SAEM_FFN_AUTO takes the one-launch step up to this many tokens (measured: faster than the five-launch
-// step at 1..4 tokens on every layer shape tried, slower at 8)
-constexpr int kDecodeFusedAutoTokens = 4;
+// SAEM_FFN_AUTO takes the one-launch step up to this many tokens (measured: 7-11 % faster than the five-launch
+// step at 1..4 tokens on every layer shape tried, level with it at 8)
+constexpr int kDecodeFusedAutoTokens = 8;
 cudaError_t launch_decode_fused(const DecodeArgs& a, const SlotTable& tab, int n_sm, cudaStream_t st, int* n_launch);
 constexpr int kDecodeSyncInts = 64 + 1024;   // d_model <= 16384: at most 1024 groups of 16 columns
 // One-time per process: resolves the driver entry point for tensor-map encoding and opts the
@@ -176,6 +183,7 @@ struct saem_ctx {
     // residency: fixed slot per (layer, expert), -1 none; temp binding per (layer, expert), -1 none
     int32_t* slot_of;        // [L*E] global slot index
     int32_t* temp_of;        // [L*E] global slot index of a temporary binding
+    const uint8_t** host_of; // [L*E] device-visible address of a packed expert in mapped pinned host memory, or null
     int32_t* slot_owner;     // [n_slots] layer*E + expert, -1 empty
     cudaEvent_t* ready_ev;   // [n_slots] recorded on the copy stream after a load
     uint8_t* ev_pending;     // [n_slots] 1: a load was enqueued and no consumer has been ordered after it yet

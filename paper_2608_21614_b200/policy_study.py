@@ -20,7 +20,7 @@ import numpy as np
 import torch
 
 from . import inputs as gen
-from .stack import StackRunner
+from .stack import StackRunner, tc_seq
 
 
 def run(trace, weights, shape, C, temp, batch, steps, policy, eap=None):
@@ -66,7 +66,8 @@ def main():
     rng = np.random.default_rng(np.random.SeedSequence([args.seed, 77]))
     weights = [gen.expert_weights(rng, cfg.d_model, cfg.d_ff) for _ in range(args.distinct)]
     full, eap = run(trace, weights, shape, cfg.n_experts, 0, args.batch, args.steps, "stage")
-    out = {"steps": args.steps, "batch": args.batch, "stages": int(len(trace.boundaries)),
+    out = {"steps": args.steps, "batch": args.batch, "layers": args.layers, "stages": int(len(trace.boundaries)),
+           "mean_stage_len": args.mean_stage_len, "tc_seq": tc_seq(eap),
            "full_gpu_tokens_per_s": full["tokens_per_s"], "runs": []}
     for ecr in [float(v) for v in args.ecr.split(",")]:
         C = max(1, int(round(ecr * cfg.n_experts)))

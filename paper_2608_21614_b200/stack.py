@@ -76,6 +76,7 @@ class StackStats:
     pair_total: int = 0
     pair_hits: int = 0
     demand_loads: int = 0
+    host_reads: int = 0        # missed experts read in place from mapped host memory
     boundary_loads: int = 0
     boundaries: int = 0
 
@@ -90,13 +91,18 @@ class StackRunner:
     def __init__(self, d_model: int, d_ff: int, n_experts: int, top_k: int, n_layers: int, slots_per_layer: int,
                  temp_slots: int, batch: int, store_weights, device: str = "cuda:0",
                  ffn_path: int = B.SAEM_FFN_AUTO, policy: str = "stage", recorded_eap: Optional[np.ndarray] = None,
-                 read_counts: bool = True):
+                 read_counts: bool = True, miss_mode: str = "temp"):
         """policy: "stage" -- at a boundary re-plan from the counts of the stage that just ended
         (the paper's online policy); "oracle" -- re-plan from `recorded_eap[s]`, the counts of the
         stage that is about to start, recorded in an earlier run of the same trace (the paper's
         clairvoyant replay, Sec. VI-D); "lru" -- no stage logic: every miss evicts the layer's least
         recently used resident expert and takes its slot (token-level baseline)."""
         assert policy in ("stage", "oracle", "lru")
+        # miss_mode: "temp" -- a missed expert is copied into a temporary slot first (the ablation's on-demand
+        # transfer); "host" -- it is bound to its pinned host buffer and the matrix-vector kernels read the
+        # weights in place over the host link (batches of at most 8 tokens): no HBM write + read, no slot.
+        assert miss_mode in ("temp", "host") and (miss_mode == "temp" or batch <= 8)
+        self.miss_mode = miss_mode
         # With every expert resident nothing on the host depends on the routing; read_counts=False
         # then skips the per-layer read-back (and with it the activation log and the hit statistics).
         self.read_counts = read_counts or slots_per_layer < n_experts
@@ -227,22 +233,32 @@ class StackRunner:
                 for e in need:                         # needs slots_per_layer >= active experts of a step
                     self._lru_load(l, e)
                 need = []
-            # every non-resident active expert must hold a temporary slot when the FFN is enqueued;
-            # a load may recycle the slot of another one of them, so repeat until all are bound
-            for _ in range(self.cfg.temp_slots + 1):
-                missing = [e for e in need if B.saem_cache_query(self.h, l, e)[0] < 0]
-                if not missing:
-                    break
-                for e in missing:
-                    self._demand_load(l, e)
+            mapped = []
+            if self.miss_mode == "host":
+                for e in need:
+                    if B.saem_cache_query(self.h, l, e)[0] < 0:
+                        B.saem_cache_map_host(self.h, l, e, self.store.get(l, e))
+                        mapped.append(e)
+                        st.host_reads += 1
+            else:
+                # every non-resident active expert must hold a temporary slot when the FFN is enqueued;
+                # a load may recycle the slot of another one of them, so repeat until all are bound
+                for _ in range(self.cfg.temp_slots + 1):
+                    missing = [e for e in need if B.saem_cache_query(self.h, l, e)[0] < 0]
+                    if not missing:
+                        break
+                    for e in missing:
+                        self._demand_load(l, e)
             self.log[l] += counts
             B.saem_expert_ffn(self.h, l, self.x_packed, self.offsets, Bt * k, active, self.y_packed)
+            for e in mapped:                           # the binding was consumed at enqueue; the host buffer stays valid
+                B.saem_cache_evict(self.h, l, e)
             B.saem_combine(self.h, self.y_packed, self.inv_perm, self.topk_w, Bt, None,
                            self.out[l] if keep_out else self.out[0])
         return self.out
 
     def h2d_bytes(self) -> int:
-        return (self.stats.demand_loads + self.stats.boundary_loads) * self.slot_bytes
+        return (self.stats.demand_loads + self.stats.boundary_loads + self.stats.host_reads) * self.slot_bytes
 
     def close(self):
         self.ctx.close()

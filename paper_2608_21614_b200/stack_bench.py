@@ -32,6 +32,8 @@ def main():
     ap.add_argument("--independent", action="store_true", help="independent ranking per stage (stress trace)")
     ap.add_argument("--trace-steps", type=int, default=4096)
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--host-reads", action="store_true",
+                    help="missed experts are read in place from mapped pinned host memory instead of being copied to a temporary slot")
     ap.add_argument("--no-readback", action="store_true",
                     help="with --ecr 1.0: do not read the routing counts back (no host sync per layer; no statistics)")
     args = ap.parse_args()
@@ -44,7 +46,7 @@ def main():
     rng = np.random.default_rng(np.random.SeedSequence([args.seed, 77]))
     weights = [gen.expert_weights(rng, d, f) for _ in range(args.distinct)]
     run = StackRunner(d, f, E, k, L, C, args.temp_slots if C < E else 0, args.batch, weights,
-                      read_counts=not args.no_readback)
+                      read_counts=not args.no_readback, miss_mode="host" if args.host_reads else "temp")
     run.warm([list(np.argsort(trace.rankings[0, l])[:C]) for l in range(L)])
     run.copy.synchronize()
     bounds = set(int(b) for b in trace.boundaries[1:])
@@ -74,7 +76,7 @@ def main():
         "trace": {"stages_seen": n_stages_seen, "tc_seq": tc_seq(stage_counts[:n_stages_seen]),
                   "kind": "independent" if args.independent else "coherent (3.2 ranks reshuffled per boundary)"},
         "chr_distinct": st.chr(), "chr_pair_weighted": st.pair_chr(), "temp_hits": st.temp_hits,
-        "demand_loads": st.demand_loads, "boundary_loads": st.boundary_loads, "boundaries": st.boundaries,
+        "demand_loads": st.demand_loads, "host_reads": st.host_reads, "miss_mode": run.miss_mode, "boundary_loads": st.boundary_loads, "boundaries": st.boundaries,
         "h2d_bytes": run.h2d_bytes(), "h2d_gbs_over_wall_time": run.h2d_bytes() / dt / 1e9,
         "slot_bytes": run.slot_bytes, "slots_per_layer": C, "temp_slots": run.cfg.temp_slots,
         "distinct_host_weight_sets": args.distinct, "device_status": B.saem_last_device_status(run.h),

@@ -108,9 +108,9 @@ def run_single_call_and_compare(layer, li, oracle, ref=None):
 
 
 # ------------------------------------------------------------------ partially resident stacks
-def run_stack(trace, weights, L, E, k, d, f, C, temp, batch, steps, keep, policy="stage", eap=None):
+def run_stack(trace, weights, L, E, k, d, f, C, temp, batch, steps, keep, policy="stage", eap=None, miss_mode="temp"):
     from paper_2608_21614_b200.stack import StackRunner
-    run = StackRunner(d, f, E, k, L, C, temp, batch, weights, policy=policy, recorded_eap=eap)
+    run = StackRunner(d, f, E, k, L, C, temp, batch, weights, policy=policy, recorded_eap=eap, miss_mode=miss_mode)
     # warm set: the C most popular experts of stage 0 (stand-in for the calibration warm-up)
     run.warm([list(np.argsort(trace.rankings[0, l])[:C]) for l in range(L)])
     outs = []

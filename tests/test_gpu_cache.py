@@ -148,3 +148,50 @@ def test_replay_policies_share_bits_and_oracle_is_no_worse(oracle):
     assert res["oracle"].hits >= res["stage"].hits
     assert res["lru"].boundary_loads == 0 and res["lru"].demand_loads > 0
     run0.close()
+
+
+def test_missed_experts_read_in_place_from_mapped_host_memory(oracle):
+    """saem_cache_map_host: an expert without a slot is bound to its packed copy in pinned host memory and
+    the matrix-vector kernels read it over the host link.  API semantics, the FFN against the oracle with
+    one expert in HBM and one in host memory, and the half-resident stack with this miss mode: identical
+    bits to full residency, the same hits as the temporary-slot mode, no on-demand copies."""
+    import gpu_util as g
+    from paper_2608_21614_b200 import binding as B
+    d, f, T = 256, 384, 6
+    wa, wb = _small_experts(2, d, f, 15)
+    ctx = B.Context(B.make_config(d, f, 2, 1, T, slots_per_layer=1, temp_slots=1))
+    h = ctx.handle
+    pa, pb = ctx.pack(*wa), ctx.pack(*wb)
+    B.saem_cache_load(h, 0, 0, 0, pa)
+    assert B.saem_cache_map_host(h, 0, 0, pb, check=False) == B.SAEM_ERR_INVALID_ARG         # has a slot
+    assert B.saem_cache_map_host(h, 0, 1, torch.empty(16, dtype=torch.uint8), check=False) == B.SAEM_ERR_INVALID_ARG   # not pinned
+    B.saem_cache_map_host(h, 0, 1, pb)
+    assert B.saem_cache_query(h, 0, 1) == (B.SAEM_HOST_MAPPED, 1)
+    rng = np.random.default_rng(4)
+    x = gen.activations(rng, T, d)
+    off = np.array([0, 2, T], np.int32)                   # rows 0..1 -> expert 0 (HBM slot), rows 2..5 -> expert 1 (host)
+    y = torch.full((T, d), float("nan"), dtype=torch.float32, device="cuda:0")
+    B.saem_expert_ffn(h, 0, g.dev(x), g.dev(off), T, None, y)
+    torch.cuda.synchronize()
+    ref = oracle.expert_ffn(x, off, [wa[0], wb[0]], [wa[1], wb[1]], [wa[2], wb[2]])
+    g.assert_close(g.host(y), ref, "one expert in HBM, one read from host memory")
+    B.saem_cache_evict(h, 0, 1)
+    assert B.saem_cache_query(h, 0, 1) == (-1, 0)
+    assert B.saem_expert_ffn(h, 0, g.dev(x), g.dev(off), T, [1], y, check=False) == B.SAEM_ERR_NOT_RESIDENT
+    assert B.saem_last_device_status(h) == 0
+    ctx.close()
+
+    L, E, k, batch, steps = 3, 8, 2, 4, 40
+    d, f = 256, 256
+    trace = gen.stage_trace(steps, L, E, 1.2, seed=11, mean_stage_len=8.0)
+    weights = _small_experts(6, d, f, 3)
+    keep = set(range(steps))
+    full, _, _, run_full = g.run_stack(trace, weights, L, E, k, d, f, E, 0, batch, steps, keep)
+    temp, st_temp, _, run_temp = g.run_stack(trace, weights, L, E, k, d, f, E // 2, 4, batch, steps, keep)
+    host, st_host, _, run_host = g.run_stack(trace, weights, L, E, k, d, f, E // 2, 4, batch, steps, keep, miss_mode="host")
+    for a, b in zip(full, host):
+        assert torch.equal(a, b)
+    assert (st_host.active, st_host.hits, st_host.boundary_loads) == (st_temp.active, st_temp.hits, st_temp.boundary_loads)
+    assert st_host.demand_loads == 0 and st_host.host_reads == st_host.active - st_host.hits > 0
+    for r in (run_full, run_temp, run_host):
+        r.close()

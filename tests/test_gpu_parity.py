@@ -254,6 +254,11 @@ def test_repack_skew_and_paper_example(oracle, B):
     rng = np.random.default_rng(2)
     cases.append((np.stack([rng.permutation(60)[:4] for _ in range(777)]).astype(np.int32), 60))
     cases.append((np.stack([rng.permutation(64)[:6] for _ in range(2048)]).astype(np.int32), 64))   # prefill size
+    # the multi-CTA index phase at its largest sizes: 128 experts top-8 at 4096 tokens (32 768 pairs), 65 535 pairs,
+    # and every pair of 40 blocks on one expert
+    cases.append((np.argsort(rng.random((4096, 128)), axis=1)[:, :8].astype(np.int32), 128))
+    cases.append((np.argsort(rng.random((13107, 64)), axis=1)[:, :5].astype(np.int32), 64))
+    cases.append((np.full((40000, 1), 5, np.int32), 9))
     for idx, E in cases:
         T, k = idx.shape
         d = 128
@@ -465,6 +470,44 @@ def test_capture_step_helper_batch_1(oracle):
     torch.cuda.synchronize()
     ref = oracle.moe_step(li2.logits, li2.x, cfg.top_k, li.gate, li.up, li.down, shared=li.shared)
     g.assert_close(g.host(layer.out[:1]), ref["out"], "graph replay, batch 1, new inputs")
+    assert layer.device_status() == 0
+    layer.close()
+
+
+def test_single_launch_step_in_a_graph_follows_new_inputs(oracle):
+    """The one-launch decode step (a cooperative launch) recorded in a CUDA graph with other steps, as a
+    decoder records its layers: replays follow new logits and activations, and the step's barrier
+    counter and tickets are left ready for the next replay."""
+    g = _g()
+    cfg = gen.LayerConfig("t", 256, 384, 60, 4, 2, 768, "zipf", 1.1, seed=17)
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, AUTO)
+    logits, x = g.dev(li.logits), g.dev(li.x)
+    out = torch.empty((2, 256), dtype=torch.float32, device="cuda:0")
+    n0 = layer.launches()
+    layer.step_fused_call(logits, x, 2, out)             # first call outside the capture
+    assert layer.launches() - n0 in (1, 2)
+    eager = out.clone()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            for _ in range(3):
+                layer.step_fused_call(logits, x, 2, out)
+    torch.cuda.current_stream().wait_stream(s)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager)
+    li2 = gen.layer_inputs(dataclasses.replace(cfg, seed=18))
+    logits.copy_(g.dev(li2.logits))
+    x.copy_(g.dev(li2.x))
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    ref = oracle.moe_step(li2.logits, li2.x, cfg.top_k, li.gate, li.up, li.down, shared=li.shared)
+    g.assert_close(g.host(out), ref["out"], "graph replay of the one-launch step on new inputs")
     assert layer.device_status() == 0
     layer.close()
 
