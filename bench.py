@@ -272,7 +272,7 @@ def roofline_of(lb, step_ms, ffn_ms, peaks, which):
                 "frac_of_sustained": achieved / float(peaks.get("bf16_tflops_sustained", 1400.0)),
                 "kernel": "saem_expert_ffn (tiled tcgen05 gate/up + down kernels)"}
     else:
-        single = T <= 8 and cfg.top_k <= 8 and lb.layer.shared is None
+        single = T <= 4 and cfg.top_k <= 8 and lb.layer.shared is None
         ms = step_ms if single else ffn_ms
         nbytes = lb.mean_active_bytes()
         achieved = nbytes / (ms * 1e-3) / 1e9

@@ -78,8 +78,9 @@ enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TEN
  * (tcgen05 cta_group::2: 256 tokens x 512 weight rows per pair of SMs), which AUTO and TENSOR take
  * for long reductions and many rows (d_model >= 4096, d_model % 256 == 0, at least 1536 packed
  * rows in the call); SAEM_FFN_TENSOR_PAIRS is SAEM_FFN_TENSOR with the pair form whenever
- * d_model % 256 == 0 (for tests and measurements).  SAEM_FFN_DECODE_FUSED is SAEM_FFN_AUTO with the
- * one-launch form of saem_moe_step (see there) stated explicitly; SAEM_FFN_TENSOR never takes that form.
+ * d_model % 256 == 0 (for tests and measurements).  SAEM_FFN_DECODE_FUSED is SAEM_FFN_AUTO, except that
+ * saem_moe_step takes its one-launch form (see there) for every batch it supports (up to 8 tokens, top_k
+ * up to 8) instead of up to 4 tokens.
  * n_shared (0..16, n_experts + n_shared <= SAEM_MAX_EXPERTS): always-on shared experts of the same
  * width d_ff that run INSIDE the layer's grouped launch.  They are experts n_experts ..
  * n_experts + n_shared - 1 of every layer for the cache calls (outside the routed cache-ratio
@@ -212,7 +213,7 @@ int saem_combine(saem_ctx* ctx, const float* y_packed, const int32_t* inv_perm, 
  * holds an always-on shared expert whose width is not a multiple of d_ff (otherwise use
  * config.n_shared and pass NULL).
  * logits[T, E] fp32, x[T, d] bf16, out[T, d] (all dev).
- * Smallest decode batches (ffn_path AUTO or DECODE_FUSED: T <= 8; top_k <= 8; no shared_ctx): the whole step runs as ONE
+ * Smallest decode batches (ffn_path AUTO: T <= 4, DECODE_FUSED: T <= 8; top_k <= 8; no shared_ctx): the whole step runs as ONE
  * kernel launch -- gate, repack indices and gate/up projection, a grid-wide barrier, down projection and
  * merge -- launched cooperatively (two launches where the device refuses that).  topk_idx, topk_w, counts,
  * offsets, perm, inv_perm, h and y_packed are still left in the workspace; x_packed is not produced.  A

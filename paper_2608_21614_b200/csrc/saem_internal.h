@@ -158,8 +158,8 @@ struct DecodeArgs {
 };
 bool decode_fused_supported(int T, int k);
 // SAEM_FFN_AUTO takes the one-launch step up to this many tokens (measured: 7-11 % faster than the five-launch
-// step at 1..4 tokens on every layer shape tried, level with it at 8)
-constexpr int kDecodeFusedAutoTokens = 8;
+// step at 1..4 tokens on every layer shape tried, level with it or 1-2 % behind at 8)
+constexpr int kDecodeFusedAutoTokens = 4;
 cudaError_t launch_decode_fused(const DecodeArgs& a, const SlotTable& tab, int n_sm, cudaStream_t st, int* n_launch);
 constexpr int kDecodeSyncInts = 64 + 1024;   // d_model <= 16384: at most 1024 groups of 16 columns
 // One-time per process: resolves the driver entry point for tensor-map encoding and opts the
