@@ -567,7 +567,11 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
     // Segments that can exceed 64 rows are a dense contraction: tile them for the tensor cores.
     // (Measured: the streaming kernels with 128-row token tiles are no faster than the tiled ones at 96 and 128
     // tokens on any of the benchmark's layer shapes, so the hand-over stays at 64 rows.)
-    if (a.n_tile > 64) {
+    // Hand-over to the tiled kernels.  Measured on whole layers (graph-replayed steps): from 17 rows per segment
+    // upwards the tiled kernels give the shorter step on every layer shape of the benchmark (1-8 % at 32..64
+    // tokens), although they pad every segment to 128 tokens -- one CTA per SM without split reductions; up to
+    // 16 rows the streaming kernels win.  SAEM_FFN_TENSOR keeps the streaming kernels up to 64 rows.
+    if (a.n_tile > a.stream_max_tile) {
         alignas(64) CUtensorMap map_h_store, map_y_store, map_x128, map_h128, map_x256, map_h256;
         if (!make_act_map(&map_x256, a.x_packed, a.max_rows, a.d, 256)) return cudaErrorInvalidValue;
         if (!make_act_map(&map_h256, a.h, a.max_rows, a.f, 256)) return cudaErrorInvalidValue;

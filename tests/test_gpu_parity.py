@@ -138,9 +138,11 @@ def test_cta_pair_tiles(oracle, T, E, k, d, f, fs):
     single.close()
 
 
-@pytest.mark.parametrize("path", [SCALAR, TENSOR], ids=["scalar", "tensor"])
+@pytest.mark.parametrize("path", [SCALAR, TENSOR, AUTO], ids=["scalar", "tensor", "auto"])
 @pytest.mark.parametrize("T,E,k,d,f,fs", [
     (1, 1, 1, 128, 128, 0),          # dense FFN, one token
+    (17, 6, 2, 256, 384, 0),         # just above the streaming kernels' 16 rows: the tiled kernels under AUTO
+    (24, 40, 4, 128, 256, 256),      # 17..64 tokens with an in-layer shared expert
     (1, 60, 4, 256, 384, 256),       # decode batch 1: four one-row segments, 56 empty, shared expert
     (9, 8, 8, 128, 256, 0),          # k == E
     (33, 60, 4, 256, 128, 0),        # E not a multiple of 32, ragged T
@@ -157,7 +159,7 @@ def test_small_shapes(oracle, path, T, E, k, d, f, fs):
     layer.close()
 
 
-@pytest.mark.parametrize("path", [SCALAR, TENSOR, PAIRS], ids=["scalar", "tensor", "cta-pairs"])
+@pytest.mark.parametrize("path", [SCALAR, TENSOR, PAIRS, AUTO], ids=["scalar", "tensor", "cta-pairs", "auto"])
 def test_segment_sizes_around_tile_edges(oracle, path):
     """One expert, k = 1: the segment is the whole batch; sizes straddle every tile boundary."""
     g = _g()
