@@ -564,15 +564,17 @@ cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream
     alignas(64) CUtensorMap map_x, map_h;
     if (!make_act_map(&map_x, a.x_packed, a.max_rows, a.d, box_rows)) return cudaErrorInvalidValue;
     if (!make_act_map(&map_h, a.h, a.max_rows, a.f, box_rows)) return cudaErrorInvalidValue;
-    // Segments that can exceed 64 rows are a dense contraction: tile them for the tensor cores.
-    // (Measured: the streaming kernels with 128-row token tiles are no faster than the tiled ones at 96 and 128
-    // tokens on any of the benchmark's layer shapes, so the hand-over stays at 64 rows.)
-    // Hand-over to the tiled kernels.  Measured on whole layers (graph-replayed steps): from 17 rows per segment
-    // upwards the tiled kernels give the shorter step on every layer shape of the benchmark (1-8 % at 32..64
-    // tokens), although they pad every segment to 128 tokens -- one CTA per SM without split reductions; up to
-    // 16 rows the streaming kernels win.  SAEM_FFN_TENSOR keeps the streaming kernels up to 64 rows.
+    // Hand-over to the tiled kernels.  Measured on whole layers (graph-replayed steps): from 9 tokens upwards the
+    // tiled kernels give the shorter step on every layer shape of the benchmark (1-8 %), although they pad every
+    // segment to 128 tokens -- one CTA per SM, whole items, no reductions across CTAs.  SAEM_FFN_AUTO therefore
+    // sends everything beyond the matrix-vector kernels' 8 rows there; SAEM_FFN_TENSOR keeps the streaming kernels
+    // up to 64 rows.
     if (a.n_tile > a.stream_max_tile) {
         alignas(64) CUtensorMap map_h_store, map_y_store, map_x128, map_h128, map_x256, map_h256;
+        if (box_rows != 32) {      // the tiled kernels load ragged token tiles as 32-row boxes, whatever the launch's tile
+            if (!make_act_map(&map_x, a.x_packed, a.max_rows, a.d, 32)) return cudaErrorInvalidValue;
+            if (!make_act_map(&map_h, a.h, a.max_rows, a.f, 32)) return cudaErrorInvalidValue;
+        }
         if (!make_act_map(&map_x256, a.x_packed, a.max_rows, a.d, 256)) return cudaErrorInvalidValue;
         if (!make_act_map(&map_h256, a.h, a.max_rows, a.f, 256)) return cudaErrorInvalidValue;
         if (!make_act_map(&map_x128, a.x_packed, a.max_rows, a.d, 128)) return cudaErrorInvalidValue;

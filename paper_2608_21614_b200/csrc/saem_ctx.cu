@@ -393,7 +393,8 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     }
     a.n_sm = c->n_sm;
     a.force_pairs = g.ffn_path == SAEM_FFN_TENSOR_PAIRS;
-    a.stream_max_tile = (g.ffn_path == SAEM_FFN_AUTO || g.ffn_path == SAEM_FFN_DECODE_FUSED) ? 16 : 64;
+    // AUTO: the tiled kernels take every launch beyond the matrix-vector kernels' 8 rows (measured on whole layers)
+    a.stream_max_tile = (g.ffn_path == SAEM_FFN_AUTO || g.ffn_path == SAEM_FFN_DECODE_FUSED) ? 0 : 64;
     int nl = 0;
     if (g.ffn_path == SAEM_FFN_SCALAR) {
         CUDA_TRY(launch_ffn_scalar(a, tab, st, &nl));

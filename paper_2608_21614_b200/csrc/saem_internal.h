@@ -129,7 +129,7 @@ struct FfnArgs {
     int max_active;             // upper bound of experts with rows: min(E, T * top_k + n_shared)
     int n_sm;
     int force_pairs;            // tiled kernels: CTA pairs whenever the shape allows
-    int stream_max_tile;        // widest token tile the streaming kernels take (16 or 64); wider launches go to the tiled kernels
+    int stream_max_tile;        // widest token tile the streaming kernels take (0: none, or 64); wider launches go to the tiled kernels
 };
 cudaError_t launch_ffn_scalar(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
 cudaError_t launch_ffn_tensor(const FfnArgs& a, const SlotTable& tab, cudaStream_t st, int* n_launch);
