@@ -49,7 +49,7 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM bytes (read + write) of the two expert-FFN kernels of one step of workload c2 at 16 tokens with all
 # 8 experts active, from an ncu capture (not measured by this run)
-NCU_FFN_TRAFFIC = {("c2", 16): (2844872000, "profiles/ffn_tensor_c2_decode.md (ncu capture, dram__bytes_read.sum + dram__bytes_write.sum)")}
+NCU_FFN_TRAFFIC = {("c2", 16): (2830469680, "profiles/ffn_prefill_c2_decode.md (ncu capture, dram__bytes_read.sum + dram__bytes_write.sum)")}
 STUDY = [("c3", 32, None), ("c3", 2048, None), ("c4", 1, None), ("c4", 8, None), ("c4", 64, None), ("c4", 8, "uniform"),
          ("c4", 64, "uniform"), ("qwen3", 1, None), ("qwen3", 8, None)]
 
@@ -158,7 +158,7 @@ def workload_name(name, cfg):
 class LayerBench:
     """One layer configuration resident on the GPU, with a few routing draws of the same stage."""
 
-    def __init__(self, name, tokens, routing, distinct, device):
+    def __init__(self, name, tokens, routing, distinct, device, ffn_path=0):
         import torch
         from paper_2608_21614_b200 import inputs as gen
         from paper_2608_21614_b200.layer import MoELayer
@@ -166,7 +166,7 @@ class LayerBench:
         self.cfg = cfg = gen.layer_config(name, tokens=tokens, routing=routing)
         self.li = li = gen.layer_inputs(cfg, n_distinct_experts=distinct)
         T, E = cfg.tokens, cfg.n_experts
-        self.layer = MoELayer(cfg.d_model, cfg.d_ff, E, cfg.top_k, T, cfg.d_ff_shared, device=device)
+        self.layer = MoELayer(cfg.d_model, cfg.d_ff, E, cfg.top_k, T, cfg.d_ff_shared, device=device, ffn_path=ffn_path)
         self.layer.load_all(li.gate, li.up, li.down, li.shared)
         self.layer.drop_host_copies()
         # The headline workload streams 2.8 GB of weights per step from one routing draw.  Smaller layers
@@ -270,7 +270,7 @@ def roofline_of(lb, step_ms, ffn_ms, peaks, which):
         roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                 "traffic": None, "algorithmic_flops": flops, "avg_ms": ffn_ms,
                 "frac_of_sustained": achieved / float(peaks.get("bf16_tflops_sustained", 1400.0)),
-                "kernel": "saem_expert_ffn (tiled tcgen05 gate/up + down kernels)"}
+                "kernel": "saem_expert_ffn (ffn_prefill_kernel<0/1>: tiled tcgen05 gate/up + down)"}
     else:
         single = T <= 4 and cfg.top_k <= 8 and lb.layer.shared is None
         ms = step_ms if single else ffn_ms
@@ -282,7 +282,9 @@ def roofline_of(lb, step_ms, ffn_ms, peaks, which):
                 "traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None,
                 "algorithmic_bytes": nbytes, "avg_ms": ms, "frac_of_nominal_8000": achieved / 8000.0,
                 "kernel": "decode_step_kernel (whole step: gate, repack indices, gate/up, down, merge in one launch)" if single
-                else "saem_expert_ffn (gate/up + down kernels%s)" % (", second call for the shared expert" if lb.layer.shared is not None else "")}
+                else "saem_expert_ffn (%s gate/up + down kernels%s)" % (
+                    "ffn_gemv_kernel<0/1>: matrix-vector" if T <= 8 else "ffn_prefill_kernel<0/1>: tiled tcgen05",
+                    ", second call for the shared expert" if lb.layer.shared is not None else "")}
     roof["peak_source"] = which
     return roof
 
@@ -382,7 +384,8 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()                                  # before warm-up: samples cover every timed region
-    lb = LayerBench(args.workload, args.tokens, args.routing, args.distinct, device)
+    lb = LayerBench(args.workload, args.tokens, args.routing, args.distinct, device,
+                    ffn_path={"auto": 0, "tensor": 2}[args.ffn_path])
     cfg = lb.cfg
     T, E, d = cfg.tokens, cfg.n_experts, cfg.d_model
     if args.graph:
@@ -475,6 +478,7 @@ def run_ours(args):
                        "routing": "%s popularity + Gumbel, seed 0" % cfg.routing, "cache": "all experts resident in HBM",
                        "l2": "layer weights %.2f GB vs 126 MB L2: inputs larger than L2, no flush" % weight_gb,
                        "distinct_weight_sets": args.distinct, "replicas": world,
+                       "ffn_path": args.ffn_path,
                        "launch": "CUDA-graph replay of the draws' steps" if args.graph else "one saem_moe_step call per step",
                        "timing": "value: K steps back to back; spread: ten more blocks; roofline: steps with events around the FFN call"},
             "spread": {"median_ms": statistics.median(blocks), "p10_ms": percentile(blocks, 0.1), "p90_ms": percentile(blocks, 0.9),
@@ -671,6 +675,8 @@ def main():
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS), help="c2 is the benchmark; the others for study")
     ap.add_argument("--tokens", type=int, default=None, help="override the batch of the workload")
     ap.add_argument("--routing", default=None, choices=["zipf", "uniform", "normal"])
+    ap.add_argument("--ffn-path", default="auto", choices=["auto", "tensor"],
+                    help="tensor: the tcgen05 weight-streaming kernels up to 64 rows per segment (SAEM_FFN_TENSOR), for comparison")
     ap.add_argument("--segments", action="store_true", help="expert-FFN throughput by segment size of one expert")
     ap.add_argument("--segment-classes", action="store_true", help="a prefill call's time by segment-size class")
     ap.add_argument("--d-model", type=int, default=2048)
