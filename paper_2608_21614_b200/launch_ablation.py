@@ -10,7 +10,7 @@ repacked batch:
               (2 launches per active expert; the host must first read the counts back)
 
 Outputs of the two modes are compared: identical bits on the matrix-vector path (no k-split), and
-equal up to fp32 summation order on the streaming path, whose k-split points depend on how many
+equal up to fp32 summation order on the streaming path (ffn_path TENSOR), whose k-split points depend on how many
 experts share the launch.
 
 With --bookkeeping the whole step is also run the way the paper describes its starting point

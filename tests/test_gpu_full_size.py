@@ -10,13 +10,15 @@ import torch
 from paper_2608_21614_b200 import inputs as gen
 
 pytestmark = pytest.mark.gpu
-TENSOR = 0      # SAEM_FFN_AUTO: the path bench.py times (matrix-vector / streaming / tiled tcgen05 by batch size)
+TENSOR = 0      # SAEM_FFN_AUTO: the path bench.py times (matrix-vector kernels up to 8 rows, tiled tcgen05 beyond)
+STREAMING = 2   # SAEM_FFN_TENSOR: the weight-streaming tcgen05 kernels up to 64 rows per segment
 
 
-def test_c2_mixtral_shaped_decode_full(oracle):
+@pytest.mark.parametrize("path", [TENSOR, STREAMING], ids=["auto-tiled", "streaming"])
+def test_c2_mixtral_shaped_decode_full(oracle, path):
     import gpu_util as g
     li = gen.layer_inputs(gen.layer_config("c2"))
-    layer = g.make_layer(li, TENSOR)
+    layer = g.make_layer(li, path)
     ref, stats = g.run_stepwise_and_compare(layer, li, oracle)
     assert int((ref["counts"] > 0).sum()) >= 6
     layer.close()
@@ -30,8 +32,12 @@ def test_fine_grained_decode_full(oracle, name, T, routing):
     import gpu_util as g
     li = gen.layer_inputs(gen.layer_config(name, tokens=T, routing=routing))
     layer = g.make_layer(li, TENSOR)
-    g.run_stepwise_and_compare(layer, li, oracle)
+    ref, _ = g.run_stepwise_and_compare(layer, li, oracle)
     layer.close()
+    if 8 < T <= 64:        # the streaming kernels at the same full size (SAEM_FFN_AUTO takes the tiled ones here)
+        layer = g.make_layer(li, STREAMING)
+        g.run_stepwise_and_compare(layer, li, oracle, ref=ref)
+        layer.close()
 
 
 @pytest.mark.parametrize("name,T", [("c4", 1), ("c4", 4), ("c4", 8), ("qwen3", 1), ("qwen3", 4), ("qwen3", 8),

@@ -141,7 +141,7 @@ def test_cta_pair_tiles(oracle, T, E, k, d, f, fs):
 @pytest.mark.parametrize("path", [SCALAR, TENSOR, AUTO], ids=["scalar", "tensor", "auto"])
 @pytest.mark.parametrize("T,E,k,d,f,fs", [
     (1, 1, 1, 128, 128, 0),          # dense FFN, one token
-    (17, 6, 2, 256, 384, 0),         # just above the streaming kernels' 16 rows: the tiled kernels under AUTO
+    (17, 6, 2, 256, 384, 0),         # 9..64 tokens: tiled kernels under AUTO, streaming kernels under TENSOR
     (24, 40, 4, 128, 256, 256),      # 17..64 tokens with an in-layer shared expert
     (1, 60, 4, 256, 384, 256),       # decode batch 1: four one-row segments, 56 empty, shared expert
     (9, 8, 8, 128, 256, 0),          # k == E
