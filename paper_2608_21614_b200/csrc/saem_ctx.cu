@@ -393,8 +393,19 @@ int saem_expert_ffn(saem_ctx* c, int layer, const void* x_packed, const int32_t*
     }
     a.n_sm = c->n_sm;
     a.force_pairs = g.ffn_path == SAEM_FFN_TENSOR_PAIRS;
-    // AUTO: the tiled kernels take every launch beyond the matrix-vector kernels' 8 rows (measured on whole layers)
-    a.stream_max_tile = (g.ffn_path == SAEM_FFN_AUTO || g.ffn_path == SAEM_FFN_DECODE_FUSED) ? 0 : 64;
+    // AUTO: the tiled kernels take every launch beyond the matrix-vector kernels' 8 rows (measured on whole layers:
+    // shorter steps on every shape) -- provided the launch can have enough whole items to occupy the SMs.  The tiled
+    // kernels deal whole (expert, 256-row weight block) items, so a launch of one or two experts (a subset, a shared
+    // expert in a context of its own) would leave most SMs idle in the down projection; the streaming kernels cut
+    // their work at k-chunk granularity and keep every SM busy.  It matters when an item is long (one Mixtral-shaped
+    // expert, d_ff 14336, at 16..64 rows: 82-102 us streaming against 127-136 us tiled); with short items the tiled
+    // kernels stay ahead even for a single expert (d_ff 1408: 30-32 us against 33-46 us).
+    {
+        const long long experts_bound = subset ? n_subset : a.max_active;
+        const bool enough_items = experts_bound * ((g.d_model + 255) / 256) * 4 >= 3LL * c->n_sm;
+        const bool auto_path = g.ffn_path == SAEM_FFN_AUTO || g.ffn_path == SAEM_FFN_DECODE_FUSED;
+        a.stream_max_tile = (auto_path && (enough_items || g.d_ff < 4096)) ? 0 : 64;
+    }
     int nl = 0;
     if (g.ffn_path == SAEM_FFN_SCALAR) {
         CUDA_TRY(launch_ffn_scalar(a, tab, st, &nl));
