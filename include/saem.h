@@ -72,7 +72,8 @@ enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TEN
  * temporary slot).  renorm: 1 = softmax over the k selected logits (weights sum to 1), 0 = the
  * selected experts' probabilities under the softmax over all experts.  out_dtype: SAEM_OUT_*.
  * ffn_path: SAEM_FFN_AUTO picks per call -- matrix-vector kernels when no segment can exceed 8
- * rows, the tcgen05 tiled kernels beyond (measured hand-over point); SAEM_FFN_TENSOR always uses the
+ * rows, the tcgen05 tiled kernels beyond (measured hand-over point; a launch of one or two experts with
+ * d_ff >= 4096 keeps the weight-streaming kernels up to 64 rows); SAEM_FFN_TENSOR always uses the
  * tcgen05 kernels: the weight-streaming ones (weights as the MMA's M operand, reductions split across
  * CTAs) up to 64 rows, the tiled ones beyond; SAEM_FFN_SCALAR forces the plain scalar
  * kernels (kept for triage).  The tiled kernels exist in two forms: one CTA per tile, and CTA pairs
