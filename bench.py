@@ -249,6 +249,21 @@ class LayerBench:
         torch.cuda.synchronize()
         return [a.elapsed_time(b) for a, b in ev]
 
+    def ffn_back_to_back(self, k):
+        """The expert-FFN call(s) of the last routing issued k times back to back (each call's set-up overlaps the
+        previous call's tail, as it overlaps the repack's inside a graph-replayed step): milliseconds per call."""
+        torch, layer, T = self.torch, self.layer, self.cfg.tokens
+        stream = torch.cuda.current_stream(self.device)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(k):
+            layer.expert_ffn(T)
+            if layer.shared is not None:
+                layer.shared_ffn(self.x, T)
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / k
+
     def close(self):
         self.layer.close()
         self.graph = None
@@ -307,7 +322,9 @@ def study_row(name, tokens, routing, distinct, device, peaks, which, min_block_m
         a, b = lb.timed_steps(k)
         torch.cuda.synchronize()
         blocks.append(a.elapsed_time(b) / k)
-    ffn = lb.ffn_pass(max(lb.n_draws * 4, 24))
+    n_ffn = max(lb.n_draws * 4, 24)
+    ffn = lb.ffn_pass(n_ffn)
+    bb_ms = lb.ffn_back_to_back(n_ffn)
     med = statistics.median(blocks)
     ffn_ms = statistics.median(ffn)
     row = {"workload": workload_name(name, cfg), "tokens_per_step": cfg.tokens, "value": cfg.tokens / (med * 1e-3), "unit": UNIT,
@@ -317,6 +334,14 @@ def study_row(name, tokens, routing, distinct, device, peaks, which, min_block_m
            "launch": "CUDA-graph replay of the draws' steps" if lb.graph is not None else "one host call per step",
            "gpu_launches_per_step": None, "roofline": roofline_of(lb, med, ffn_ms, peaks, which),
            "device_status": lb.layer.device_status()}
+    roof = row["roofline"]
+    if "decode_step_kernel" not in roof["kernel"]:
+        if roof["bound"] == "hbm":      # bytes of the draw that call ran on (the last one of the instrumented pass)
+            bb = (lb.active[(n_ffn - 1) % lb.n_draws] * lb.weight_bytes + lb.shared_bytes) / (bb_ms * 1e-3) / 1e9
+        else:
+            bb = roof["achieved"] * ffn_ms / bb_ms
+        roof["back_to_back"] = {"avg_ms": bb_ms, "achieved": bb, "frac": bb / roof["peak"],
+                                "note": "the same saem_expert_ffn call issued back to back on one routing draw"}
     n0 = lb.layer.launches()
     lb.step(0)
     row["gpu_launches_per_step"] = lb.layer.launches() - n0
@@ -424,17 +449,7 @@ def run_ours(args):
     # timed region 2: steps with CUDA events around the saem_expert_ffn call(s) -> the dominant kernels' duration
     ffn_ms = lb.ffn_pass(max(K, 24))
     # the same call issued back to back on the last routing (its set-up overlaps the previous call's tail)
-    bb0, bb1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    Kb = min(max(K, 24), 200)
-    stream = torch.cuda.current_stream()
-    bb0.record(stream)
-    for _ in range(Kb):
-        lb.layer.expert_ffn(T)
-        if lb.layer.shared is not None:
-            lb.layer.shared_ffn(lb.x, T)
-    bb1.record(stream)
-    torch.cuda.synchronize()
-    ffn_bb_ms = bb0.elapsed_time(bb1) / Kb
+    ffn_bb_ms = lb.ffn_back_to_back(min(max(K, 24), 200))
     status = lb.layer.device_status()
 
     # end to end through the host-buffer call: H2D of logits and x, the kernels, D2H of out
