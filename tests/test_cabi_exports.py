@@ -64,3 +64,22 @@ def test_weight_packer_is_a_permutation_of_the_input_bytes():
     # the matching up tile follows the gate tile
     tile_u = out[128 * 64:2 * 128 * 64].reshape(128, 8, 8)
     assert np.array_equal(tile_u[5, 2 ^ 5], up[5, 16:24])
+
+
+def test_header_constants_match_the_binding_and_large_repack_shapes_are_accepted():
+    """The enumerators of include/saem.h have the values the ctypes binding uses, and the shapes that the
+    one-CTA repack index phase used to refuse (128 experts top-8 beyond 2560 tokens) are valid configs."""
+    from paper_2608_21614_b200 import binding as B
+    text = open(os.path.join(ROOT, "include", "saem.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    consts = dict((k, int(v)) for k, v in re.findall(r"\b(SAEM_[A-Z0-9_]+)\s*=\s*(-?\d+)\s*[,}]", text))
+    consts["SAEM_STATIC_SCRATCH_ELEMS"] = 1 << 20                                  # written as 1 << 20 in the header
+    assert re.search(r"SAEM_STATIC_SCRATCH_ELEMS\s*=\s*1\s*<<\s*20", text)
+    assert len(consts) >= 20
+    for name, value in consts.items():
+        assert getattr(B, name) == value, name
+    for E, k, T in ((128, 8, 4096), (64, 5, 13107), (9, 1, 40000)):
+        cfg = B.make_config(128, 128, E, k, T)
+        assert B.saem_slot_bytes(cfg) > 0 and B.saem_workspace_bytes(cfg) > 0
+    assert B.saem_slot_bytes(B.make_config(128, 128, 64, 5, 13108)) == 0          # 65 540 pairs: one too many tokens
+    assert B.make_config(128, 128, 8, 2, 4, ffn_path=B.SAEM_FFN_DECODE_FUSED).ffn_path == 4
