@@ -201,14 +201,12 @@ class StackRunner:
         Bt, k = self.batch, self.k
         st = self.stats
         for l in range(self.L):
+            if not self.read_counts:                   # nothing on the host depends on the routing: the single call
+                B.saem_moe_step(self.h, None, l, logits_all[l], x, Bt, self.out[l] if keep_out else self.out[0])
+                continue
             B.saem_route(self.h, logits_all[l], Bt, self.topk_idx, self.topk_w)
             B.saem_repack(self.h, self.topk_idx, x, Bt, self.counts, self.offsets, self.perm, self.inv_perm,
                           self.x_packed)
-            if not self.read_counts:
-                B.saem_expert_ffn(self.h, l, self.x_packed, self.offsets, Bt * k, None, self.y_packed)
-                B.saem_combine(self.h, self.y_packed, self.inv_perm, self.topk_w, Bt, None,
-                               self.out[l] if keep_out else self.out[0])
-                continue
             self.counts_host.copy_(self.counts, non_blocking=True)
             self.counts_ready.record(self.compute)
             self.counts_ready.synchronize()

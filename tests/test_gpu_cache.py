@@ -195,3 +195,31 @@ def test_missed_experts_read_in_place_from_mapped_host_memory(oracle):
     assert st_host.demand_loads == 0 and st_host.host_reads == st_host.active - st_host.hits > 0
     for r in (run_full, run_temp, run_host):
         r.close()
+
+
+@pytest.mark.parametrize("batch", [2, 12])
+def test_fully_resident_stack_without_readback_uses_the_single_call(oracle, batch):
+    """With every expert resident nothing on the host depends on the routing: read_counts=False drives each
+    layer through the single saem_moe_step call (the one-launch decode step at batch 2), with no host
+    synchronisation per layer.  Every layer-step against the oracle."""
+    import gpu_util as g
+    from paper_2608_21614_b200.stack import StackRunner
+    L, E, k, d, f, steps = 3, 8, 2, 256, 384, 5
+    trace = gen.stage_trace(steps, L, E, 1.2, seed=21, mean_stage_len=3.0)
+    weights = _small_experts(5, d, f, 8)
+    run = StackRunner(d, f, E, k, L, E, 0, batch, weights, read_counts=False)
+    assert not run.read_counts
+    run.warm([list(range(E)) for _ in range(L)])
+    for t in range(steps):
+        lg = np.stack([gen.trace_logits(trace, t, l, batch) for l in range(L)])
+        x = gen.trace_activations(trace, t, batch, d)
+        out = run.step(torch.from_numpy(lg).cuda(), torch.from_numpy(x).cuda())
+        torch.cuda.synchronize()
+        for l in range(L):
+            ws = [run.store.weights(l, e) for e in range(E)]
+            ref = oracle.moe_step(lg[l], x, k, [w[0] for w in ws], [w[1] for w in ws], [w[2] for w in ws])
+            g.assert_close(g.host(out[l]), ref["out"], "step %d layer %d" % (t, l))
+    from paper_2608_21614_b200 import binding as B
+    assert B.saem_last_device_status(run.h) == 0
+    assert run.stats.layer_steps == 0                     # no read-back, hence no statistics
+    run.close()
