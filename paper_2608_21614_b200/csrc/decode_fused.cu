@@ -208,7 +208,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
     extern __shared__ __align__(16) uint8_t ring_raw[];
     __shared__ DecodeIndex sm;
     __shared__ float red[kDfWarps][8][32];
-    __shared__ int head_unit[kDfWarps];
+    __shared__ int head_units[2][kDfWarps];           // per phase
     __shared__ __align__(8) uint64_t stage_bar[kDfWarps][kDfStages];
     __shared__ int barrier_ok, abort_flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -318,7 +318,8 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
     // `requested` chunks have been requested by the caller already.  Complete tiles are delivered through `finish`,
     // partial ones parked.  Returns false if a wait ran out.
     uint32_t parity = 0;                               // bit s: the phase of stage s's barrier to wait for next
-    auto stream = [&](auto unit_tag, const WarpWork& ww, int KC, int upe, auto& finish, int requested) -> bool {
+    auto stream = [&](auto unit_tag, const WarpWork& ww, int KC, int upe, auto& finish, int requested, int* head_unit,
+                      auto&& after_loop) -> bool {
         using U = decltype(unit_tag);
         // ---- producer state (lane 0 issues) ----
         int pu = ww.u0, pkc = ww.kc0, pleft = ww.n;
@@ -432,6 +433,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
                 run = in_unit;
             }
         }
+        after_loop();                                  // this warp's ring is free again
         __syncthreads();
         if (ok && tail_unit >= 0 && !abort_flag) {     // add the following warps' heads in warp order
             for (int w2 = warp + 1; w2 < kDfWarps && head_unit[w2] == tail_unit; ++w2)
@@ -442,33 +444,36 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
         return ok;
     };
 
+    // Phase B's deal and the request of its first weight stages: a warp does this the moment its own phase-A
+    // loop is over (or at once in a phase-B-only launch), before it meets its CTA and the grid.
+    const int KC_b = a.f / kTileK, upe_b = a.d / 32;
+    WarpWork ww_b = {0, 0, 0, 1};
+    int requested_b = 0;
+    auto prefetch_b = [&]() {
+        ww_b = deal_units(n_active * upe_b, KC_b, warp);
+        if (lane == 0) head_units[1][warp] = -1;
+        int pu = ww_b.u0, pkc = ww_b.kc0;
+        for (; requested_b < kDfStages && requested_b < ww_b.n; ++requested_b) {
+            if (lane == 0) {
+                const uint32_t dst = ring + (uint32_t)requested_b * kDfStageBytes, bar = bars + 8u * requested_b;
+                mbar_expect_tx(bar, 4096u);
+                bulk_g2s(dst, Unit<1>::weights(a, tab, sm, pu, upe_b, KC_b) + (size_t)pkc * Unit<1>::kStride, 4096, bar);
+            }
+            if (++pkc == KC_b) { pu += ww_b.ustep; pkc = 0; }
+        }
+    };
+
     // ================================ phase A: gate/up + SiLU*mul ================================
     if (phase_mask & 1) {
         const int KC = a.d / kTileK, upe = a.f / 16;
         const WarpWork ww = deal_units(n_active * upe, KC, warp);
-        if (lane == 0) head_unit[warp] = -1;
-        stream(Unit<0>(), ww, KC, upe, finish_a, 0);
+        if (lane == 0) head_units[0][warp] = -1;
+        stream(Unit<0>(), ww, KC, upe, finish_a, 0, head_units[0], [&]() { if (phase_mask & 2) prefetch_b(); });
     }
 
     // ================================ phase B: down + merge ================================
     if (phase_mask & 2) {
-        const int KC = a.f / kTileK, upe = a.d / 32;
-        const WarpWork ww = deal_units(n_active * upe, KC, warp);
-        if (phase_mask == 3) __syncthreads();          // phase A's readers of head_unit are done
-        if (lane == 0) head_unit[warp] = -1;
-        // weights of the first stages go out before this warp meets the grid (or waits for the phase-A launch)
-        int requested = 0;
-        {
-            int pu = ww.u0, pkc = ww.kc0;
-            for (; requested < kDfStages && requested < ww.n; ++requested) {
-                if (lane == 0) {
-                    const uint32_t dst = ring + (uint32_t)requested * kDfStageBytes, bar = bars + 8u * requested;
-                    mbar_expect_tx(bar, 4096u);
-                    bulk_g2s(dst, Unit<1>::weights(a, tab, sm, pu, upe, KC) + (size_t)pkc * Unit<1>::kStride, 4096, bar);
-                }
-                if (++pkc == KC) { pu += ww.ustep; pkc = 0; }
-            }
-        }
+        if (!(phase_mask & 1)) prefetch_b();
         bool ok = true;
         if (phase_mask == 3) {
             // Grid barrier: every h store of phase A is visible device-wide before anyone reads h.  The CTA's
@@ -499,7 +504,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             pdl_wait();                                // h is complete from here on
             pdl_launch_dependents();
         }
-        if (ok) stream(Unit<1>(), ww, KC, upe, finish_b, requested);
+        if (ok) stream(Unit<1>(), ww_b, KC_b, upe_b, finish_b, requested_b, head_units[1], []() {});
     }
     // Copies still in flight (a wait that ran out, a barrier that was not met) must land before the CTA's shared
     // memory goes away.
