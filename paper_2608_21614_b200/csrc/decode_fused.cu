@@ -366,33 +366,42 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
         int stage = 0;
         bool ok = true;
         const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+        // Activation pieces travel through registers, fetched two chunks ahead of the MMAs that use them: the fetch
+        // cursor (unit, chunks left in it, chunks left in the range) runs ahead of the consumer's own.
         const uint16_t* xq = nullptr;                  // this lane's activation row at the chunk to be fetched next
-        uint4 xa = zero4, xb = zero4;                  // activation pieces of the current chunk
+        int au = u, a_run = KC - kc_begin, a_left = left;
         if (left > 0) {
             xq = U::acts(a, sm, u, upe, g, t);
+            if (xq) xq += (size_t)kc_begin * kTileK;
+        }
+        auto fetch = [&](uint4& pa, uint4& pb) {
+            pa = zero4;
+            pb = zero4;
+            if (a_left <= 0) return;
+            if (a_run == 0) {                          // the next chunk opens the range's next unit
+                au += ww.ustep;
+                xq = U::acts(a, sm, au, upe, g, t);
+                a_run = KC;
+            }
             if (xq) {
-                xq += (size_t)kc_begin * kTileK;
-                xa = ld_act(xq);
-                xb = ld_act(xq + 32);
+                pa = ld_act(xq);
+                pb = ld_act(xq + 32);
                 xq += kTileK;
             }
-        }
+            --a_run;
+            --a_left;
+        };
+        uint4 xa, xb, na, nb;                          // pieces of the current chunk and of the one after it
+        fetch(xa, xb);
+        fetch(na, nb);
         // this lane's weight pieces inside a stage: rows g (+ 8 per set) of the first 2 KB, the matching rows 2 KB further
         // (up rows in phase A; rows + 16 ... in phase B the second set is 2 KB further and the + 8 rows 1 KB further)
         const uint32_t w_lo = ring + (uint32_t)g * 128u;
         constexpr uint32_t kSetStep = U::kStride == 2u * kTileBytes ? 1024u : 2048u;     // bytes from set 0's rows g to set 1's
         constexpr uint32_t kHiStep = U::kStride == 2u * kTileBytes ? 2048u : 1024u;      // bytes from rows g to the set's rows g + 8
         while (left > 0) {
-            // activation pieces of the next chunk (it may belong to the next unit of this range)
-            uint4 na = zero4, nb = zero4;
-            if (left > 1) {
-                if (run == 1) xq = U::acts(a, sm, u + ww.ustep, upe, g, t);
-                if (xq) {
-                    na = ld_act(xq);
-                    nb = ld_act(xq + 32);
-                    xq += kTileK;
-                }
-            }
+            uint4 ma, mb;                              // pieces of the chunk after the next one
+            fetch(ma, mb);
             ok = mbar_wait(bars + 8u * stage, (parity >> stage) & 1u, &abort_flag, a.status, kDfBarrierLimitNs);
             if (!ok) break;
             parity ^= 1u << stage;
@@ -412,6 +421,8 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             if (++stage == kDfStages) stage = 0;
             xa = na;
             xb = nb;
+            na = ma;
+            nb = mb;
             --left;
             if (--run == 0) {                          // this range's share of unit u is complete
                 if (kc_begin > 0) {                    // started inside the unit: a head partial
