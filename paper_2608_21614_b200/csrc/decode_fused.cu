@@ -211,6 +211,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
     __shared__ int head_units[2][kDfWarps];           // per phase
     __shared__ __align__(8) uint64_t stage_bar[kDfWarps][kDfStages];
     __shared__ int barrier_ok, abort_flag;
+    __shared__ unsigned long long barrier_target;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;            // MMA fragment coordinates
     const int P = a.T * a.k, ES = a.E + a.S;
@@ -230,8 +231,9 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
         pdl_wait();
         pdl_launch_dependents();
     }
-    unsigned long long barrier_target = 0;
-    if (phase_mask == 3 && tid == 0) {                // before this CTA arrives, the counter cannot pass the next multiple of G
+    // Before this CTA arrives, the barrier counter cannot pass the next multiple of G.  The last warp reads it (warp 0
+    // is on the critical path: it routes token 0) and leaves the target in shared memory for thread 0.
+    if (phase_mask == 3 && tid == kDfThreads - 32) {
         unsigned long long c;
         asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(c) : "l"(a.sync) : "memory");
         barrier_target = (c / gridDim.x + 1ull) * gridDim.x;
@@ -460,7 +462,40 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
     const int KC_b = a.f / kTileK, upe_b = a.d / 32;
     WarpWork ww_b = {0, 0, 0, 1};
     int requested_b = 0;
+    // Column form of phase B, for the very smallest steps (at most 16 active experts, d_model / 16 <= grid): CTA j
+    // owns output columns 16 j .. 16 j + 15 of EVERY active expert, a warp is (expert, part of the reduction
+    // length), and the merge over a token's experts happens in this CTA's shared memory: no ticket, no read-back of
+    // y through L2 (two to three dependent L2 round trips at the end of a step that is all latency).  A stage holds
+    // the unit's 16 rows of two consecutive chunks (2 KB each).
+    const int n_pairs_b = KC_b >> 1;
+    const bool columns_b = n_active <= kDfWarps && (a.d >> 4) <= (int)gridDim.x;     // (d_ff is a multiple of 128: KC_b is even)
+    int cw_ks = 1, cw_ai = 0, cw_p0 = 0, cw_n = 0, cw_left = 0;     // warps per expert; this warp's expert, first pair, pairs; pairs not requested yet
+    const uint8_t* cw_wp = nullptr;                                 // weights of the next pair to request
+    auto request_pair = [&](int stage) {
+        if (lane == 0) {
+            const uint32_t dst = ring + (uint32_t)stage * kDfStageBytes, bar = bars + 8u * stage;
+            mbar_expect_tx(bar, 4096u);
+            bulk_g2s(dst, cw_wp, 2048, bar);
+            bulk_g2s(dst + 2048, cw_wp + kTileBytes, 2048, bar);
+        }
+        cw_wp += 2 * (size_t)kTileBytes;
+        --cw_left;
+    };
     auto prefetch_b = [&]() {
+        if (columns_b) {
+            while (n_active * cw_ks * 2 <= kDfWarps && cw_ks * 2 <= n_pairs_b) cw_ks *= 2;
+            cw_ai = warp / cw_ks;
+            const int part = warp % cw_ks, j = (int)blockIdx.x;
+            if (cw_ai < n_active && j < (a.d >> 4)) {
+                cw_p0 = n_pairs_b * part / cw_ks;
+                cw_n = n_pairs_b * (part + 1) / cw_ks - cw_p0;
+                cw_wp = a.slot_region + (size_t)tab.slot[sm.act[cw_ai]] * a.slot_bytes + (size_t)2 * a.d * a.f * 2 +
+                        ((size_t)(j >> 3) * KC_b + 2 * cw_p0) * kTileBytes + (size_t)(j & 7) * 2048u;
+            }
+            cw_left = cw_n;
+            for (; requested_b < kDfStages && requested_b < cw_n; ++requested_b) request_pair(requested_b);
+            return;
+        }
         ww_b = deal_units(n_active * upe_b, KC_b, warp);
         if (lane == 0) head_units[1][warp] = -1;
         int pu = ww_b.u0, pkc = ww_b.kc0;
@@ -472,6 +507,84 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             }
             if (++pkc == KC_b) { pu += ww_b.ustep; pkc = 0; }
         }
+    };
+    // The column form's streaming and merge; every thread of the CTA calls it.  Returns false if a wait ran out.
+    auto columns_phase_b = [&]() -> bool {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        bool ok = true;
+        if (cw_n > 0) {
+            const int e = sm.act[cw_ai];
+            const uint16_t* hq = g < sm.counts[e] ? a.h + (size_t)(sm.offsets[e] + g) * a.f + (size_t)cw_p0 * (2 * kTileK) + t * 8
+                                                  : nullptr;
+            const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+            uint4 x[4] = {zero4, zero4, zero4, zero4};             // pieces of the current pair: k 8t.., 32 + 8t.., 64 + 8t.., 96 + 8t..
+            if (hq) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) x[q] = ld_act(hq + 32 * q);
+                hq += 2 * kTileK;
+            }
+            const uint32_t w_lo = ring + (uint32_t)g * 128u;
+            int stage = 0;
+            for (int i = 0; i < cw_n; ++i) {
+                uint4 nx[4] = {zero4, zero4, zero4, zero4};
+                if (i + 1 < cw_n && hq) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) nx[q] = ld_act(hq + 32 * q);
+                    hq += 2 * kTileK;
+                }
+                ok = mbar_wait(bars + 8u * stage, (parity >> stage) & 1u, &abort_flag, a.status, kDfBarrierLimitNs);
+                if (!ok) break;
+                parity ^= 1u << stage;
+                const uint32_t base = w_lo + (uint32_t)stage * kDfStageBytes;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {                        // the pair's two chunks: rows g and g + 8 of each
+                    const uint32_t lo = base + (uint32_t)c * 2048u, hi = lo + 1024u;
+                    const uint4 w00 = ld_shared_v4(lo + piece0), w01 = ld_shared_v4(lo + piece1);
+                    const uint4 w10 = ld_shared_v4(hi + piece0), w11 = ld_shared_v4(hi + piece1);
+                    mma_16816(acc, w00.x, w10.x, w00.y, w10.y, x[2 * c].x, x[2 * c].y);
+                    mma_16816(acc, w00.z, w10.z, w00.w, w10.w, x[2 * c].z, x[2 * c].w);
+                    mma_16816(acc, w01.x, w11.x, w01.y, w11.y, x[2 * c + 1].x, x[2 * c + 1].y);
+                    mma_16816(acc, w01.z, w11.z, w01.w, w11.w, x[2 * c + 1].z, x[2 * c + 1].w);
+                }
+                __syncwarp();
+                if (cw_left > 0) request_pair(stage);
+                if (++stage == kDfStages) stage = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) x[q] = nx[q];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) red[warp][i][lane] = acc[i];
+        __syncthreads();
+        if (abort_flag || (int)blockIdx.x >= (a.d >> 4)) return ok && !abort_flag;
+        // Merge: thread (token, column) adds the token's experts in slot order, shared experts last (the combine
+        // kernel's arithmetic); an expert's value is the sum of its warps' partial tiles in warp order.  Accumulator
+        // fragment: element 2 * (column / 8) + (row & 1) of lane 4 * (column & 7) + row / 2, row = the token's row
+        // inside the expert's segment.
+        for (int o = tid; o < a.T * 16; o += kDfThreads) {
+            const int tok = o >> 4, c = o & 15, col = (int)blockIdx.x * 16 + c;
+            auto value = [&](int e, int r) -> float {
+                int ai = 0;
+                while (sm.act[ai] != e) ++ai;
+                const int ln = (c & 7) * 4 + (r >> 1), fi = (c >> 3) * 2 + (r & 1);
+                float v = red[ai * cw_ks][fi][ln];
+                for (int q = 1; q < cw_ks; ++q) v += red[ai * cw_ks + q][fi][ln];
+                a.y_packed[(size_t)(sm.offsets[e] + r) * a.d + col] = v;
+                return v;
+            };
+            float s = 0.f;
+            for (int jj = 0; jj < a.k; ++jj) {
+                const int e = sm.idx[tok * a.k + jj];
+                if (tab.slot[e] < 0) continue;
+                s = fmaf(sm.w[tok * a.k + jj], value(e, sm.inv[tok * a.k + jj] - sm.offsets[e]), s);
+            }
+            for (int sh = 0; sh < a.S; ++sh)
+                if (tab.slot[a.E + sh] >= 0) s += value(a.E + sh, tok);
+            const size_t at = (size_t)tok * a.d + col;
+            if (a.out_bf16) reinterpret_cast<__nv_bfloat16*>(a.out)[at] = __float2bfloat16_rn(s);
+            else reinterpret_cast<float*>(a.out)[at] = s;
+        }
+        return ok;
     };
 
     // ================================ phase A: gate/up + SiLU*mul ================================
@@ -496,11 +609,12 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
                 int good = abort_flag ? 0 : 1;
                 unsigned long long* counter = reinterpret_cast<unsigned long long*>(a.sync);
                 asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(counter) : "memory");
+                const unsigned long long target = barrier_target;
                 unsigned long long t0 = 0;
                 for (uint32_t i = 0;; ++i) {
                     unsigned long long c;
                     asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(c) : "l"(counter) : "memory");
-                    if (c >= barrier_target) break;
+                    if (c >= target) break;
                     if ((i & 255u) == 255u) {
                         const unsigned long long now = globaltimer_ns();
                         if (t0 == 0) t0 = now;
@@ -515,7 +629,10 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             pdl_wait();                                // h is complete from here on
             pdl_launch_dependents();
         }
-        if (ok) stream(Unit<1>(), ww_b, KC_b, upe_b, finish_b, requested_b, head_units[1], []() {});
+        if (ok) {
+            if (columns_b) columns_phase_b();
+            else stream(Unit<1>(), ww_b, KC_b, upe_b, finish_b, requested_b, head_units[1], []() {});
+        }
     }
     // Copies still in flight (a wait that ran out, a barrier that was not met) must land before the CTA's shared
     // memory goes away.
