@@ -13,10 +13,12 @@
 //            SiLU*mul happens in the accumulator registers of one thread and nothing is exchanged
 //            between warps.  Token rows are read straight from x through the permutation (no x_packed).
 //   phase B  y = Wd h for 32 output columns of one active expert per warp unit, then the merge (Sec.
-//            IV-D): each group of 32 columns has a ticket counter, and the warp that delivers a
-//            group's last expert adds the k contributions of every token in slot order j = 0..k-1,
+//            IV-D): each (group of 32 columns, token) has a ticket counter, and the warp that delivers
+//            a token's last contribution adds the token's k contributions in slot order j = 0..k-1,
 //            shared experts last, with the arithmetic of the combine kernel (deterministic whoever
-//            does it; nobody waits for anybody).
+//            does it; nobody waits for anybody; the merges are spread over the whole phase).  With at
+//            most 16 active experts a CTA owns 16 columns of every expert instead and merges them in
+//            its own shared memory.
 //
 // Between the phases the grid meets at a barrier (a cooperative launch guarantees that all CTAs are
 // resident; the wait is bounded and gives up with SAEM_ERR_TIMEOUT).  Before it arrives, every warp
@@ -49,6 +51,7 @@ constexpr int kDfStages = 3;
 constexpr int kDfStageBytes = 4096;              // per warp and stage: the 32 weight rows of one chunk of a unit
 constexpr int kDfRingBytes = kDfWarps * kDfStages * kDfStageBytes + 128;
 constexpr unsigned long long kDfBarrierLimitNs = 200000000ull;   // 0.2 s
+constexpr int kDfTicketOff = 64;               // the step's synchronisation words: barrier counter, then the merge's tickets
 
 struct DecodeIndex {
     int32_t idx[kDfMaxPairs];
@@ -59,6 +62,7 @@ struct DecodeIndex {
     int32_t offsets[SAEM_MAX_EXPERTS + 1];
     int16_t act[SAEM_MAX_EXPERTS];          // experts with rows AND a slot, ascending id
     int warp_act[4];
+    int need[kDfMaxTokens];                 // contributions a token's merge waits for: its resident experts + resident shared ones
     int n_active;
     int absent;                             // an expert with rows has no slot
 };
@@ -130,6 +134,13 @@ __device__ __forceinline__ void build_index(const DecodeArgs& a, const SlotTable
         const int r = sm.offsets[e] + rank;
         sm.perm[r] = tid;
         sm.inv[tid] = r;
+    }
+    if (tid >= kDfThreads - a.T) {
+        const int tok = kDfThreads - 1 - tid;
+        int n = 0;
+        for (int j = 0; j < a.k; ++j) n += tab.slot[sm.idx[tok * a.k + j]] >= 0 ? 1 : 0;
+        for (int sh = 0; sh < a.S; ++sh) n += tab.slot[a.E + sh] >= 0 ? 1 : 0;
+        sm.need[tok] = n;
     }
     __syncthreads();
 }
@@ -270,7 +281,7 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             if (2 * t + 1 < m) hb[(size_t)(row0 + 2 * t + 1) * a.f + col] = __float2bfloat16_rn(c[1] / (1.f + expf(-c[1])) * c[3]);
         }
     };
-    auto finish_b = [&](int u, const float* acc) {    // store y, take a ticket for the 32 columns, merge them if last
+    auto finish_b = [&](int u, const float* acc) {    // store y, take the tokens' tickets for the 32 columns, merge what is complete
         const int upe = a.d / 32;
         const int ai = u / upe, j = u - ai * upe;
         const int e = sm.act[ai], row0 = sm.offsets[e], m = sm.counts[e];
@@ -290,25 +301,42 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
         }
         __threadfence();
         __syncwarp();
-        int last = 0;
-        if (lane == 0) {
-            int* ticket = a.sync + 64 + j;
-            last = atomicAdd(ticket, 1) == n_active - 1;
+        // One ticket per (column group, token): lane r < m speaks for the token of the segment's row r.  The warp that
+        // delivers a token's last contribution merges that token's 32 columns (lane = column): the k values are
+        // requested together, then added in slot order with fused multiply-adds, shared experts last -- the combine
+        // kernel's arithmetic, whoever does it.
+        int tok = 0;
+        bool last = false;
+        if (lane < m) {
+            tok = e < a.E ? sm.perm[row0 + lane] / a.k : lane;
+            int* ticket = a.sync + kDfTicketOff + j * kDfMaxTokens + tok;
+            last = atomicAdd(ticket, 1) == sm.need[tok] - 1;
             if (last) *ticket = 0;                     // every contributor has arrived: ready for the next step
         }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (!last) return;
+        unsigned done = __ballot_sync(0xffffffffu, last);
+        if (!done) return;
         __threadfence();
-        for (int o = lane; o < a.T * 32; o += 32) {
-            const int tok = o >> 5, c = o & 31;
-            float s = 0.f;
-            for (int jj = 0; jj < a.k; ++jj) {         // slot order, fused multiply-adds: the combine kernel's arithmetic
-                if (tab.slot[sm.idx[tok * a.k + jj]] < 0) continue;
-                s = fmaf(sm.w[tok * a.k + jj], __ldcg(y + (size_t)sm.inv[tok * a.k + jj] * a.d + j * 32 + c), s);
+        const float* yc = y + j * 32 + lane;
+        while (done) {
+            const int tk = __shfl_sync(0xffffffffu, tok, __ffs(done) - 1);
+            done &= done - 1;
+            float v[kDfMaxK];
+            unsigned present = 0;
+#pragma unroll
+            for (int jj = 0; jj < kDfMaxK; ++jj) {
+                v[jj] = 0.f;
+                if (jj < a.k && tab.slot[sm.idx[tk * a.k + jj]] >= 0) {
+                    v[jj] = __ldcg(yc + (size_t)sm.inv[tk * a.k + jj] * a.d);
+                    present |= 1u << jj;
+                }
             }
+            float s = 0.f;
+#pragma unroll
+            for (int jj = 0; jj < kDfMaxK; ++jj)
+                if (present >> jj & 1u) s = fmaf(sm.w[tk * a.k + jj], v[jj], s);
             for (int sh = 0; sh < a.S; ++sh)
-                if (tab.slot[a.E + sh] >= 0) s += __ldcg(y + (size_t)(P + sh * a.T + tok) * a.d + j * 32 + c);
-            const size_t at = (size_t)tok * a.d + j * 32 + c;
+                if (tab.slot[a.E + sh] >= 0) s += __ldcg(yc + (size_t)(P + sh * a.T + tk) * a.d);
+            const size_t at = (size_t)tk * a.d + j * 32 + lane;
             if (a.out_bf16) reinterpret_cast<__nv_bfloat16*>(a.out)[at] = __float2bfloat16_rn(s);
             else reinterpret_cast<float*>(a.out)[at] = s;
         }
@@ -630,8 +658,20 @@ decode_step_kernel(DecodeArgs a, const __grid_constant__ SlotTable tab, int phas
             pdl_launch_dependents();
         }
         if (ok) {
-            if (columns_b) columns_phase_b();
-            else stream(Unit<1>(), ww_b, KC_b, upe_b, finish_b, requested_b, head_units[1], []() {});
+            if (columns_b) {
+                columns_phase_b();
+            } else {
+                if (blockIdx.x == 0) {                 // a token without any resident expert gets no ticket: its output is zero
+                    for (int tok = 0; tok < a.T; ++tok) {
+                        if (sm.need[tok] > 0) continue;
+                        for (int c = tid; c < a.d; c += kDfThreads) {
+                            if (a.out_bf16) reinterpret_cast<__nv_bfloat16*>(a.out)[(size_t)tok * a.d + c] = __float2bfloat16_rn(0.f);
+                            else reinterpret_cast<float*>(a.out)[(size_t)tok * a.d + c] = 0.f;
+                        }
+                    }
+                }
+                stream(Unit<1>(), ww_b, KC_b, upe_b, finish_b, requested_b, head_units[1], []() {});
+            }
         }
     }
     // Copies still in flight (a wait that ran out, a barrier that was not met) must land before the CTA's shared

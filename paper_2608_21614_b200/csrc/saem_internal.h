@@ -31,7 +31,7 @@ struct SlotTable {
 struct WorkspaceLayout {
     size_t status;        // int32 status word (+ padding)
     size_t counters;      // int32[2 * kMaxCtas] split-K arrival counters (gate/up, down)
-    size_t decode_sync;   // int32[kDecodeSyncInts] grid barrier and column-group tickets of the one-launch decode step
+    size_t decode_sync;   // int32[kDecodeSyncInts] grid barrier and (column group, token) tickets of the one-launch decode step
     size_t h;             // bf16 [max_rows, d_ff]
     size_t partials;      // fp32 [CTAs][2][2][n_tile][128]: 2 CTAs/SM for n_tile <= 64, else 1 CTA/SM
     size_t repack_hist;   // int32 [64][SAEM_MAX_EXPERTS] per-block histograms of the multi-CTA repack
@@ -162,7 +162,7 @@ bool decode_fused_supported(int T, int k);
 // step at 1..4 tokens on every layer shape tried, level with it or 1-2 % behind at 8)
 constexpr int kDecodeFusedAutoTokens = 4;
 cudaError_t launch_decode_fused(const DecodeArgs& a, const SlotTable& tab, int n_sm, cudaStream_t st, int* n_launch);
-constexpr int kDecodeSyncInts = 64 + 1024;   // d_model <= 16384: at most 1024 groups of 16 columns
+constexpr int kDecodeSyncInts = 64 + 4096;   // d_model <= 16384: at most 512 groups of 32 columns, a ticket per group and token (<= 8)
 // One-time per process: resolves the driver entry point for tensor-map encoding and opts the
 // kernels into large dynamic shared memory.  Returns cudaSuccess or the failing error.
 cudaError_t ffn_tensor_init();

@@ -113,6 +113,35 @@ def test_single_launch_decode_step_bf16_out_and_absent_expert(oracle, B):
     layer.close()
 
 
+@pytest.mark.parametrize("T,E,k", [(8, 64, 4), (2, 8, 2)])
+def test_single_launch_step_token_without_any_resident_expert(oracle, B, T, E, k):
+    """None of token 0's experts has a slot: its output row is zero, the other tokens' rows merge what
+    is resident, the status word says NOT_RESIDENT.  The first case has more than 16 active experts
+    (merge by tickets), the second at most 16 (merge inside the CTA that owns the columns)."""
+    g = _g()
+    cfg = gen.LayerConfig("t", 256, 256, E, k, T, 0, "uniform", seed=77)
+    li = gen.layer_inputs(cfg, n_distinct_experts=min(E, 6))
+    ref = oracle.moe_step(li.logits, li.x, k, li.gate, li.up, li.down)
+    missing = set(int(e) for e in ref["topk_idx"][0])
+    from paper_2608_21614_b200.layer import MoELayer
+    layer = MoELayer(256, 256, E, k, T, ffn_path=FUSED)
+    for e in range(E):
+        if e not in missing:
+            layer.load_expert(0, e, e, li.gate[e], li.up[e], li.down[e])
+    o = torch.full((T, 256), 7.0, dtype=torch.float32, device="cuda:0")
+    layer.step_fused_call(g.dev(li.logits), g.dev(li.x), T, o)
+    torch.cuda.synchronize()
+    assert layer.device_status() == B.SAEM_ERR_NOT_RESIDENT
+    gate, up, down = list(li.gate), list(li.up), list(li.down)
+    for e in missing:
+        gate[e], up[e], down[e] = np.zeros_like(gate[e]), np.zeros_like(up[e]), np.zeros_like(down[e])
+    ref2 = oracle.moe_step(li.logits, li.x, k, gate, up, down)
+    out = g.host(o)
+    assert not out[0].any()
+    g.assert_close(out, ref2["out"], "tokens beside the one without a resident expert")
+    layer.close()
+
+
 @pytest.mark.parametrize("T,E,k,d,f,fs", [
     (300, 8, 2, 256, 256, 0),        # one pair of weight blocks in gate/up, a single block in down
     (700, 12, 3, 512, 384, 384),     # odd number of f-blocks (a one-block item), in-layer shared expert, ragged tiles
