@@ -17,9 +17,18 @@
 //     copy warp's loads).  Each epilogue warp therefore stages its 32 rows x 64 bytes in shared
 //     memory (64-byte swizzle, conflict-free) and hands them to the TMA as one tile store; only the
 //     ragged last rows of a segment are stored directly, row by row.
-//   * One persistent CTA per SM; whole tiles are dealt round-robin in the order (expert, weight
-//     block, token tile), so the CTAs that run at the same time share a weight block and it is
-//     fetched from HBM once and re-read from L2.  No tile is split, nothing is reduced across CTAs.
+//   * One persistent CTA per SM; whole tiles are dealt in the order (expert, weight block, token
+//     tile), so the CTAs that run at the same time share a weight block and it is fetched from HBM
+//     once and re-read from L2.  No tile is split, nothing is reduced across CTAs.
+//   * The two launches overlap at their seam.  The gate/up launch deals its items round-robin, and
+//     its last, partial round keeps a few SMs busy for one more item (an item alone on an SM is
+//     bound by the latency of its K / 64 stages, not by bytes: 25 us on the Mixtral shape) while
+//     all the others are done.  The down launch therefore does not wait for the whole gate/up grid
+//     (programmatic dependent launch without the wait): its CTAs start on the SMs that grid has
+//     left, take their items from a counter in the same order (late starters get less), and wait
+//     per expert -- bounded -- for a count of that expert's completed h rows, which the gate/up
+//     epilogue warps advance item by item.  Experts complete in ascending order, so only the items
+//     of the last expert ever wait.  The counts are put back to zero by their last reader.
 //   * 128 or 256 tokens per item is decided per launch on the device: a stage is released only
 //     when its MMAs have completed and its refill takes about a microsecond, so with 4 x 48 KB
 //     stages of 128-token items the tensor pipe idles about a third of the time; two token tiles
@@ -44,6 +53,7 @@ struct PfPlan {
     int total_items;
     int tpi;                // tokens per item: 128 or 256
     int slot[SAEM_MAX_EXPERTS];
+    int eid[SAEM_MAX_EXPERTS];      // expert id of the active expert
     int row0[SAEM_MAX_EXPERTS];
     int rows[SAEM_MAX_EXPERTS];
     int item_base[SAEM_MAX_EXPERTS + 1];
@@ -82,6 +92,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
     __shared__ __align__(8) uint64_t bar_full[kPfMaxStages], bar_empty[kPfMaxStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
+    __shared__ int claimed[16];            // down launch: the items this CTA has claimed, in order (-1: no more)
     __shared__ int s_warp_act[kPfThreads / 32], s_warp_t1[kPfThreads / 32], s_warp_t2[kPfThreads / 32];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -102,8 +113,18 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    pdl_wait();
+    // The gate/up launch waits for whatever produced its inputs.  The down launch does NOT wait for the whole
+    // gate/up grid: it starts on the SMs that grid has left (all of its CTAs have passed their own wait by then, so
+    // everything older is complete) and waits per expert for that expert's h rows (counters below), so the last
+    // gate/up items -- a partial round on a few SMs -- overlap the down projection of the other experts.
+    if (PHASE == 0) pdl_wait();
     pdl_launch_dependents();
+    // a.counters[e]: token rows x f-blocks of expert e whose h is complete, counted once per epilogue warp (8 x f-blocks
+    // x rows when all of it is there); a.counters[kMaxCtas + e]: down items of expert e that have seen that.  The last
+    // of those puts both back to zero for the next call.
+    int* const h_ready = a.counters;
+    int* const h_seen = a.counters + kMaxCtas;
+    int* const next_item = a.counters + 2 * kMaxCtas;      // down launch: the next unclaimed item
 
     // ---- plan (one thread per expert, block-wide prefix sums) ----
     {
@@ -146,6 +167,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         if (rows > 0) {
             const int n = base_act + act_inc - 1;
             plan.slot[n] = tab.slot[e];
+            plan.eid[n] = e;
             plan.row0[n] = r0;
             plan.rows[n] = rows;
             plan.item_base[n] = pair ? (base_t2 + t2_inc - t2) * WB : (base_t1 + t1_inc - t1) * WB;
@@ -167,12 +189,36 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
 
     if (warp == 0) {
         // =============================== producer ===============================
-        int stage = 0, cursor = 0;
+        int stage = 0, cursor = 0, ready_a = -1;
         uint32_t phase = 0;
         bool ok = true;
         int issued = 0;
         PfItem it;
-        for (int item = blockIdx.x; ok && item < total_items; item += G) {
+        // Gate/up: whole items round-robin.  Down: items are claimed in the same order with one atomic add each, because
+        // this launch's CTAs start at different times -- the SMs of the gate/up launch's last round join late and must
+        // get less.  The G failing claims at the end put the counter back to zero.
+        auto claim = [&]() -> int {
+            int v = 0;
+            if (lane == 0) {
+                v = atomicAdd(next_item, 1);
+                if (v == total_items + G - 1) *next_item = 0;
+            }
+            return v;
+        };
+        int upcoming = PHASE == 0 ? (int)blockIdx.x : claim();
+        for (int n = 0; ok; ++n) {
+            const int item = __shfl_sync(0xffffffffu, upcoming, 0);
+            if (item >= total_items) {
+                if (PHASE == 1) {               // tell the MMA warp through the next stage's barrier
+                    ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, a.status);
+                    if (ok && lane == 0) {
+                        claimed[n & 15] = -1;
+                        mbar_arrive(smem_u32(&bar_full[stage]));
+                    }
+                }
+                break;
+            }
+            if (PHASE == 1 && lane == 0) claimed[n & 15] = item;
             pf_decode(plan, item, cursor, WB, last_cols, it);
             const uint8_t* slot = a.slot_region + (size_t)plan.slot[it.a] * a.slot_bytes;
             // gate/up: chunk (f-block, kc) is 32 KB (gate tile, up tile); down: tiles (2 wb, kc), (2 wb + 1, kc)
@@ -182,6 +228,21 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             const size_t w_step = PHASE == 0 ? kPfStageW : kTileBytes;
             const int n_boxes = (it.rows_here + 31) / 32;
             const uint32_t w_bytes = it.n_cols == 256 ? kPfStageW : kTileBytes;
+            if (PHASE == 1) {       // this expert's h must be complete; every item says that it has seen it
+                const int e = plan.eid[it.a];
+                int good = 1;
+                if (lane == 0) {
+                    if (it.a != ready_a) good = counter_wait(h_ready + e, 8 * (a.f / kTileRows) * plan.rows[it.a], abort_p, a.status) ? 1 : 0;
+                    if (good && atomicAdd(h_seen + e, 1) == plan.item_base[it.a + 1] - plan.item_base[it.a] - 1) {
+                        h_ready[e] = 0;
+                        h_seen[e] = 0;
+                    }
+                    fence_proxy_async_all();
+                }
+                ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+                if (!ok) break;
+                ready_a = it.a;
+            }
             for (int kc = 0; kc < KC; ++kc) {
                 ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, a.status);
                 if (!ok) break;
@@ -210,6 +271,9 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 ++issued;
                 if (++stage == n_stages) { stage = 0; phase ^= 1u; }
             }
+            // the next item: claimed only now, with this item's last stages still in flight -- a CTA never holds an item
+            // it is not yet working on, so that a launch of fewer items than CTAs gives each CTA at most one
+            upcoming = PHASE == 0 ? item + G : claim();
         }
         if (!ok && issued > 0) {     // let copies already in flight land before the CTA's memory goes away
             unsigned long long t0 = globaltimer_ns();
@@ -221,12 +285,27 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         uint32_t phase = 0, acc_phase[2] = {0u, 0u};
         bool ok = true;
         PfItem it;
-        for (int item = blockIdx.x; ok && item < total_items; item += G) {
+        for (int n = 0; ok; ++n) {
+            int item = blockIdx.x + n * G;
+            if (PHASE == 0 && item >= total_items) break;
+            ok = mbar_wait(smem_u32(&bar_full[stage]), phase, abort_p, a.status);     // the item's first stage
+            if (!ok) break;
+            if (PHASE == 1) {                    // which item it is was written before the stage was requested
+                item = claimed[n & 15];
+                if (item < 0) {
+                    // No more items: pass it on to the epilogue warps through the barrier of the accumulator that the next
+                    // tile would have used -- once they have taken that accumulator's previous tile (a barrier must not
+                    // complete two phases before its waiters have seen the first), and behind the MMAs still in flight.
+                    ok = mbar_wait(smem_u32(&bar_acc_empty[acc]), acc_phase[acc] ^ 1u, abort_p, a.status);
+                    if (ok && lane == 0) tc_commit(smem_u32(&bar_acc_full[acc]));
+                    break;
+                }
+            }
             pf_decode(plan, item, cursor, WB, last_cols, it);
             const int acc0 = acc, acc1 = acc ^ 1;             // accumulators of the item's first / second tile
             const uint32_t idesc = idesc_bf16(it.n_cols);
             for (int kc = 0; ok && kc < KC; ++kc) {
-                ok = mbar_wait(smem_u32(&bar_full[stage]), phase, abort_p, a.status);
+                if (kc > 0) ok = mbar_wait(smem_u32(&bar_full[stage]), phase, abort_p, a.status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t ws = smem_base + (uint32_t)stage * stage_bytes;
@@ -271,11 +350,19 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         uint32_t acc_phase[2] = {0u, 0u};
         bool ok = true;
         PfItem it;
-        for (int item = blockIdx.x; ok && item < total_items; item += G) {
+        for (int n = 0; ok; ++n) {
+            int item = blockIdx.x + n * G;
+            if (PHASE == 0 && item >= total_items) break;
+            ok = mbar_wait(smem_u32(&bar_acc_full[acc]), acc_phase[acc], abort_p, a.status);     // the item's first tile
+            if (!ok) break;
+            if (PHASE == 1) {
+                item = claimed[n & 15];
+                if (item < 0) break;
+            }
             pf_decode(plan, item, cursor, WB, last_cols, it);
             for (int t = 0; ok && t < it.n_mt; ++t) {
                 const int ac = t == 0 ? acc : acc ^ 1;
-                ok = mbar_wait(smem_u32(&bar_acc_full[ac]), acc_phase[ac], abort_p, a.status);
+                if (t > 0) ok = mbar_wait(smem_u32(&bar_acc_full[ac]), acc_phase[ac], abort_p, a.status);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ac * 256);
@@ -372,6 +459,12 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 }
             }
             if (it.n_mt == 1) acc ^= 1;
+            if (PHASE == 0 && ok) {                 // this warp's share of the item's h is complete and visible device-wide
+                if (lane == 0) { bulk_wait_all(); fence_proxy_async_all(); }
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(h_ready + plan.eid[it.a], it.rows_here);
+            }
         }
         if (lane == 0) bulk_wait_all();         // this warp's tile stores have landed
     }

@@ -42,7 +42,7 @@ WorkspaceLayout workspace_layout(const saem_config& c) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, A); return o; };
     L.status = take(256);
-    L.counters = take(sizeof(int) * 2 * kMaxCtas);
+    L.counters = take(sizeof(int) * (2 * kMaxCtas + 16));
     L.decode_sync = take(sizeof(int) * kDecodeSyncInts);
     L.h = take(R * f * 2);
     {   // split-K partial tiles of the streaming kernels: token tiles of at most 64 rows, two slots per CTA

@@ -30,7 +30,8 @@ struct SlotTable {
 
 struct WorkspaceLayout {
     size_t status;        // int32 status word (+ padding)
-    size_t counters;      // int32[2 * kMaxCtas] split-K arrival counters (gate/up, down)
+    size_t counters;      // int32[2 * kMaxCtas + 16] split-K arrival counters (gate/up, down) of the streaming kernels; the tiled
+                          // kernels keep per-expert "h complete" / "seen" counts and the down launch's item counter there
     size_t decode_sync;   // int32[kDecodeSyncInts] grid barrier and (column group, token) tickets of the one-launch decode step
     size_t h;             // bf16 [max_rows, d_ff]
     size_t partials;      // fp32 [CTAs][2][2][n_tile][128]: 2 CTAs/SM for n_tile <= 64, else 1 CTA/SM
@@ -122,7 +123,7 @@ struct FfnArgs {
     uint16_t* h;                // [max_rows, f] bf16 workspace
     float* y_packed;            // [max_rows, d]
     int* status;
-    int* counters;              // [2 * kMaxCtas]
+    int* counters;              // [2 * kMaxCtas + 16]
     float* partials;
     size_t partial_slot_floats;
     int n_tile;                 // token tile for this launch (multiple of 16, <= 256)

@@ -81,6 +81,29 @@ __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.w
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // orders this thread's ordinary shared-memory writes before later async-proxy (TMA) reads of them
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// orders this thread's generic-proxy accesses (flags, fences) against its async-proxy (TMA) accesses to global memory
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// Bounded wait until a device-wide counter has reached `need` (acquire).  False, abort flag and SAEM_ERR_TIMEOUT
+// if it has not within the limit, or if the CTA has given up elsewhere.
+__device__ __forceinline__ bool counter_wait(const int* ctr, int need, volatile int* abort_flag, int* status,
+                                             unsigned long long limit_ns = kWaitLimitNs) {
+    unsigned long long t0 = 0;
+    for (uint32_t i = 0;; ++i) {
+        int c;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(c) : "l"(ctr) : "memory");
+        if (c >= need) return true;
+        if ((i & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) {
+                *abort_flag = 1;
+                atomicExch(status, SAEM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }

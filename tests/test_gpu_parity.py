@@ -577,6 +577,53 @@ def test_empty_batch_and_limits(B):
     ctx.close()
 
 
+@pytest.mark.parametrize("T,path", [(8, AUTO), (48, AUTO), (48, TENSOR), (700, AUTO)])
+def test_ffn_counters_are_zero_between_calls(oracle, T, path):
+    """Every counter through which the FFN kernels' CTAs meet (split-item arrivals of the streaming
+    kernels; per-expert completion counts and the item counter of the tiled kernels, whose down launch
+    starts while the gate/up launch's last items still run) is back at zero after each call, and a
+    second step on other inputs is as correct as the first."""
+    g = _g()
+    cfg = gen.LayerConfig("t", 512, 384, 12, 3, T, 384, "zipf", 1.1, seed=5 + T)
+    li = gen.layer_inputs(cfg)
+    layer = g.make_layer(li, path)
+    counters = layer.ctx.step_tensor(10, (656,), torch.int32)
+    for seed in (5 + T, 905 + T):
+        li2 = gen.layer_inputs(dataclasses.replace(cfg, seed=seed))
+        li2 = dataclasses.replace(li2, gate=li.gate, up=li.up, down=li.down, shared=li.shared)
+        g.run_stepwise_and_compare(layer, li2, oracle)
+        torch.cuda.synchronize()
+        assert int(counters.abs().sum()) == 0
+    layer.close()
+
+
+@pytest.mark.parametrize("T,E,k,d,f,fs", [(1500, 16, 2, 256, 640, 0), (2048, 64, 6, 256, 384, 768), (40, 8, 2, 512, 1024, 0)])
+def test_tiled_kernels_many_calls_in_a_row(oracle, T, E, k, d, f, fs):
+    """Several hundred steps and expert-FFN calls in a row on the tiled kernels (two-tile items whose
+    epilogue runs behind the MMAs; a down launch that starts while the gate/up launch still runs and
+    takes its items from a counter): no wait ever runs out, every counter is back at zero, and the
+    output of every step is bit-identical to the first one's."""
+    g = _g()
+    cfg = gen.LayerConfig("t", d, f, E, k, T, fs, "zipf", 1.1, seed=11 * T + E)
+    li = gen.layer_inputs(cfg, n_distinct_experts=min(E, 6))
+    layer = g.make_layer(li, AUTO)
+    g.run_stepwise_and_compare(layer, li, oracle)
+    logits, x = g.dev(li.logits), g.dev(li.x)
+    first = layer.step(logits, x, T).clone()
+    counters = layer.ctx.step_tensor(10, (656,), torch.int32)
+    for rep in range(6):
+        for _ in range(50):
+            out = layer.step(logits, x, T)
+        for _ in range(50):
+            layer.expert_ffn(T)
+        layer.combine(T)
+        torch.cuda.synchronize()
+        assert layer.device_status() == 0
+        assert int(counters.abs().sum()) == 0
+        assert torch.equal(out, first)
+    layer.close()
+
+
 def test_bounded_device_wait_runs_out_and_context_survives(oracle, B):
     """Failure detection without a GPU fault: a wait that nothing will ever satisfy gives up after
     its limit, the kernel returns, the status word says TIMEOUT, and the same context then runs a
@@ -587,10 +634,11 @@ def test_bounded_device_wait_runs_out_and_context_survives(oracle, B):
     layer = g.make_layer(li, TENSOR)
     # a CTA that gives up a wait skips its arrival on a split item's counter; stand in for that on the
     # host by leaving a count behind, and check that reading the TIMEOUT status clears the counters
-    counters = layer.ctx.step_tensor(10, (640,), torch.int32)
+    counters = layer.ctx.step_tensor(10, (656,), torch.int32)
     assert int(counters.abs().sum()) == 0
     counters[3] = 2
     counters[320 + 17] = 1
+    counters[640] = 5
     t0 = time.perf_counter()
     B.saem_selftest_bounded_wait(layer.ctx.handle, 20000)            # 20 ms limit
     torch.cuda.synchronize()
