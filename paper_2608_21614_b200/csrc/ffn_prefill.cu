@@ -28,7 +28,9 @@
 //     left, take their items from a counter in the same order (late starters get less), and wait
 //     per expert -- bounded -- for a count of that expert's completed h rows, which the gate/up
 //     epilogue warps advance item by item.  Experts complete in ascending order, so only the items
-//     of the last expert ever wait.  The counts are put back to zero by their last reader.
+//     of the last expert ever wait.  The counts are put back to zero by their last reader.  (Only
+//     when the down projection has more than one round of items; with a single round the overlap
+//     gains nothing and the down launch waits for the gate/up grid as a whole.)
 //   * 128 or 256 tokens per item is decided per launch on the device: a stage is released only
 //     when its MMAs have completed and its refill takes about a microsecond, so with 4 x 48 KB
 //     stages of 128-token items the tensor pipe idles about a third of the time; two token tiles
@@ -53,6 +55,7 @@ struct PfPlan {
     int total_items;
     int tpi;                // tokens per item: 128 or 256
     int x_bytes;            // token rows of a stage: as many 32-row boxes as the launch's longest item has
+    int seam;               // the down launch overlaps the gate/up launch's last round (both launches take the same decision)
     int slot[SAEM_MAX_EXPERTS];
     int eid[SAEM_MAX_EXPERTS];      // expert id of the active expert
     int row0[SAEM_MAX_EXPERTS];
@@ -114,10 +117,11 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // The gate/up launch waits for whatever produced its inputs.  The down launch does NOT wait for the whole
-    // gate/up grid: it starts on the SMs that grid has left (all of its CTAs have passed their own wait by then, so
-    // everything older is complete) and waits per expert for that expert's h rows (counters below), so the last
-    // gate/up items -- a partial round on a few SMs -- overlap the down projection of the other experts.
+    // The gate/up launch waits for whatever produced its inputs.  The down launch does not, at this point: it starts on
+    // the SMs that the gate/up grid has left (all of that grid's CTAs have passed their own wait by then, so everything
+    // older is complete), makes its plan, and then either waits for the whole gate/up grid (a single round of down
+    // items, see the plan) or waits per expert for that expert's h rows (counters below), so that the last gate/up
+    // items -- a partial round on a few SMs -- overlap the down projection of the other experts.
     if (PHASE == 0) pdl_wait();
     pdl_launch_dependents();
     // a.counters[e]: token rows x f-blocks of expert e whose h is complete, counted once per epilogue warp (8 x f-blocks
@@ -181,6 +185,11 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             plan.n_active = tot_act;
             plan.total_items = (pair ? tot_t2 : tot_t1) * WB;
             plan.tpi = pair ? 256 : 128;
+            // Overlapping the launches pays when the down projection has more than one round of items: with a single
+            // round (the Mixtral shape at 16 tokens: 128 items of 7 MB) the items that wait for the last expert's h
+            // are as long as the whole launch, nothing is gained and the shared bandwidth stretches the gate/up tail
+            // (measured 1 % slower), so the down launch then simply waits for the gate/up grid.
+            plan.seam = (long long)tot_t1 * ((a.d / kTileRows + 1) / 2) > (long long)gridDim.x ? 1 : 0;
             int longest = 0;
             for (int w = 0; w < kPfThreads / 32; ++w) longest = max(longest, s_warp_max[w]);
             if (longest > plan.tpi) longest = plan.tpi;
@@ -188,6 +197,8 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         }
         __syncthreads();
     }
+    const bool seam = plan.seam != 0;
+    if (PHASE == 1 && !seam) pdl_wait();        // (the plan above read only what was complete before the gate/up launch began)
     const uint32_t tmem_base = tmem_base_s;
     const int total_items = plan.total_items;
     // A stage: 32 KB of weights, then the token rows: 16 KB per 128-token tile (four stages of 48 KB, or three of
@@ -213,7 +224,8 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         // Gate/up: whole items round-robin.  Down: items are claimed in the same order with one atomic add each, because
         // this launch's CTAs start at different times -- the SMs of the gate/up launch's last round join late and must
         // get less.  The G failing claims at the end put the counter back to zero.
-        auto claim = [&]() -> int {
+        auto claim = [&](int after) -> int {
+            if (!seam) return after + G;            // every CTA starts at the same time: round-robin
             int v = 0;
             if (lane == 0) {
                 v = atomicAdd(next_item, 1);
@@ -221,7 +233,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             }
             return v;
         };
-        int upcoming = PHASE == 0 ? (int)blockIdx.x : claim();
+        int upcoming = PHASE == 0 || !seam ? (int)blockIdx.x : claim(0);
         for (int n = 0; ok; ++n) {
             const int item = __shfl_sync(0xffffffffu, upcoming, 0);
             if (item >= total_items) {
@@ -244,7 +256,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             const size_t w_step = PHASE == 0 ? kPfStageW : kTileBytes;
             const int n_boxes = (it.rows_here + 31) / 32;
             const uint32_t w_bytes = it.n_cols == 256 ? kPfStageW : kTileBytes;
-            if (PHASE == 1) {       // this expert's h must be complete; every item says that it has seen it
+            if (PHASE == 1 && seam) {       // this expert's h must be complete; every item says that it has seen it
                 const int e = plan.eid[it.a];
                 int good = 1;
                 if (lane == 0) {
@@ -289,7 +301,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             }
             // the next item: claimed only now, with this item's last stages still in flight -- a CTA never holds an item
             // it is not yet working on, so that a launch of fewer items than CTAs gives each CTA at most one
-            upcoming = PHASE == 0 ? item + G : claim();
+            upcoming = PHASE == 0 ? item + G : claim(item);
         }
         if (!ok && issued > 0) {     // let copies already in flight land before the CTA's memory goes away
             unsigned long long t0 = globaltimer_ns();
@@ -475,7 +487,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 }
             }
             if (it.n_mt == 1) acc ^= 1;
-            if (PHASE == 0 && ok) {                 // this warp's share of the item's h is complete and visible device-wide
+            if (PHASE == 0 && seam && ok) {         // this warp's share of the item's h is complete and visible device-wide
                 if (lane == 0) { bulk_wait_all(); fence_proxy_async_all(); }
                 __threadfence();
                 __syncwarp();
