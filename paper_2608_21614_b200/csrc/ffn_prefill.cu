@@ -29,8 +29,9 @@
 //     per expert -- bounded -- for a count of that expert's completed h rows, which the gate/up
 //     epilogue warps advance item by item.  Experts complete in ascending order, so only the items
 //     of the last expert ever wait.  The counts are put back to zero by their last reader.  (Only
-//     when the down projection has more than one round of items; with a single round the overlap
-//     gains nothing and the down launch waits for the gate/up grid as a whole.)
+//     where it pays -- see the plan: more than one round of down items, and long segments or a
+//     gate/up launch whose last round leaves at least half of the SMs idle; otherwise the down
+//     launch waits for the gate/up grid as a whole.)
 //   * 128 or 256 tokens per item is decided per launch on the device: a stage is released only
 //     when its MMAs have completed and its refill takes about a microsecond, so with 4 x 48 KB
 //     stages of 128-token items the tensor pipe idles about a third of the time; two token tiles
@@ -44,7 +45,7 @@ namespace saem {
 constexpr int kPfThreads = 320;            // warp 0 copies, warp 1 MMA, warps 2..9 epilogue
 constexpr int kPfStageW = 2 * kTileBytes;  // 256 weight rows x 64 k
 constexpr int kPfTileX = 128 * 128;        // one 128-token tile x 64 k
-constexpr int kPfMaxStages = 5;
+constexpr int kPfMaxStages = 4;
 constexpr int kPfStageArea = 4 * (kPfStageW + kPfTileX);     // = 3 x (32 KB + 2 x 16 KB) as well
 constexpr int kPfStoreBuf = 2048;          // per epilogue warp: 32 rows x 64 bytes on their way out
 constexpr int kPfSmem = kPfStageArea + 8 * kPfStoreBuf + 1024;
@@ -54,7 +55,6 @@ struct PfPlan {
     int n_active;
     int total_items;
     int tpi;                // tokens per item: 128 or 256
-    int x_bytes;            // token rows of a stage: as many 32-row boxes as the launch's longest item has
     int seam;               // the down launch overlaps the gate/up launch's last round (both launches take the same decision)
     int slot[SAEM_MAX_EXPERTS];
     int eid[SAEM_MAX_EXPERTS];      // expert id of the active expert
@@ -96,8 +96,8 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
     __shared__ __align__(8) uint64_t bar_full[kPfMaxStages], bar_empty[kPfMaxStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
-    __shared__ int claimed[16];            // down launch: the items this CTA has claimed, in order (-1: no more)
-    __shared__ int s_warp_act[kPfThreads / 32], s_warp_t1[kPfThreads / 32], s_warp_t2[kPfThreads / 32], s_warp_max[kPfThreads / 32];
+    __shared__ int claimed[16];            // down launch with claimed items: this CTA's items in order (-1: no more, -2: not known yet)
+    __shared__ int s_warp_act[kPfThreads / 32], s_warp_t1[kPfThreads / 32], s_warp_t2[kPfThreads / 32];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int K = PHASE == 0 ? a.d : a.f;
@@ -107,6 +107,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
     const int last_cols = PHASE == 0 ? 256 : ((a.d / kTileRows) & 1 ? 128 : 256);
     const uint32_t smem_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
 
+    if (tid < 16) claimed[tid] = -2;
     if (tid == 0) {
         abort_flag = 0;
         for (int s = 0; s < kPfMaxStages; ++s) { mbar_init(smem_u32(&bar_full[s]), 1); mbar_init(smem_u32(&bar_empty[s]), 1); }
@@ -154,10 +155,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                       n2 = __shfl_up_sync(0xffffffffu, t2_inc, o);
             if (lane >= o) { act_inc += na; t1_inc += n1; t2_inc += n2; }
         }
-        int rows_max = rows;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) rows_max = max(rows_max, __shfl_xor_sync(0xffffffffu, rows_max, o));
-        if (lane == 31) { s_warp_act[warp] = act_inc; s_warp_t1[warp] = t1_inc; s_warp_t2[warp] = t2_inc; s_warp_max[warp] = rows_max; }
+        if (lane == 31) { s_warp_act[warp] = act_inc; s_warp_t1[warp] = t1_inc; s_warp_t2[warp] = t2_inc; }
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
@@ -185,15 +183,22 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             plan.n_active = tot_act;
             plan.total_items = (pair ? tot_t2 : tot_t1) * WB;
             plan.tpi = pair ? 256 : 128;
-            // Overlapping the launches pays when the down projection has more than one round of items: with a single
-            // round (the Mixtral shape at 16 tokens: 128 items of 7 MB) the items that wait for the last expert's h
-            // are as long as the whole launch, nothing is gained and the shared bandwidth stretches the gate/up tail
-            // (measured 1 % slower), so the down launch then simply waits for the gate/up grid.
-            plan.seam = (long long)tot_t1 * ((a.d / kTileRows + 1) / 2) > (long long)gridDim.x ? 1 : 0;
-            int longest = 0;
-            for (int w = 0; w < kPfThreads / 32; ++w) longest = max(longest, s_warp_max[w]);
-            if (longest > plan.tpi) longest = plan.tpi;
-            plan.x_bytes = ((longest + 31) / 32) * 4096;
+            // Do the two launches overlap at their seam?  (Both launches take this decision, from the same numbers.)
+            //  * Not when the down projection is a single round of items (the Mixtral shape at 16 tokens: 128 items of
+            //    7 MB): the items that wait for the last expert's h are as long as the whole launch, nothing is gained
+            //    and the shared bandwidth stretches the gate/up tail (measured 1 % slower).
+            //  * When the segments are long (prefill: the SMs that the gate/up launch's last round leaves idle are idle
+            //    tensor pipes), always.
+            //  * When they are short (decode: weight streaming) only if that last round occupies at most half of the SMs:
+            //    a fuller round keeps HBM busy by itself, and the overlap's bookkeeping then costs more than the idle SMs
+            //    could have fetched (c3 at 32 tokens, 106 of 148 SMs in the last round: 1 % slower with the overlap; the
+            //    Qwen3 shape at 16 tokens, 64 of 148: 5 % faster).
+            const int G = (int)gridDim.x;
+            const int wb_gu = a.f / kTileRows, wb_down = (a.d / kTileRows + 1) / 2;
+            const bool pair_gu = 2ll * tot_t2 * wb_gu >= (long long)kPfPairHalfRounds * G && 2 * tot_t1 >= 3 * tot_t2;
+            const int rest_gu = (int)(((long long)(pair_gu ? tot_t2 : tot_t1) * wb_gu) % G);
+            const bool long_segments = 2 * tot_t1 >= 3 * tot_act;
+            plan.seam = (long long)tot_t1 * wb_down > (long long)G && (long_segments || (rest_gu != 0 && 2 * rest_gu <= G)) ? 1 : 0;
         }
         __syncthreads();
     }
@@ -201,18 +206,26 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
     if (PHASE == 1 && !seam) pdl_wait();        // (the plan above read only what was complete before the gate/up launch began)
     const uint32_t tmem_base = tmem_base_s;
     const int total_items = plan.total_items;
-    // A stage: 32 KB of weights, then the token rows: 16 KB per 128-token tile (four stages of 48 KB, or three of
-    // 64 KB with two tiles per item).  An MMA always reads a whole 128-row tile, whatever the item's rows.  Where the
-    // reduction is short (at most 32 stages per item) and no item has more than 32 rows (decode), the token rows get
-    // only the 4 KB they need and a fifth stage fits: an item's first refills are a visible part of such an item
-    // (measured: 2 % of the step on the layers with d_model 2048).  The MMA then reads on into the next stage's
-    // weights -- rows of the accumulator that are never stored.  Long reductions stream; there the packed layout
-    // was measured 0.5 % slower (Mixtral shape), so they keep the plain one.
-    const bool packed_rows = KC <= 32 && plan.x_bytes == 4096;
-    const uint32_t stage_bytes = kPfStageW + (packed_rows ? 4096u : (uint32_t)(plan.tpi / 128) * kPfTileX);
-    const int n_stages = packed_rows ? 5 : (plan.tpi == 128 ? 4 : 3);
+    const int n_stages = plan.tpi == 128 ? 4 : 3;
+    const uint32_t stage_bytes = kPfStageW + (uint32_t)(plan.tpi / 128) * kPfTileX;
     const int G = gridDim.x;
     volatile int* abort_p = &abort_flag;
+    // The copy warp publishes each claimed item in `claimed` as soon as it knows it; the other warps read it there before
+    // the item's first stage has arrived (bounded: -3 if the CTA has given up).
+    auto claimed_item = [&](int n) -> int {
+        const volatile int* slot = &claimed[n & 15];
+        unsigned long long t0 = 0;
+        for (uint32_t i = 0;; ++i) {
+            const int v = *slot;
+            if (v != -2) return v;
+            if ((i & 1023u) == 1023u) {
+                if (*abort_p) return -3;
+                const unsigned long long now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kWaitLimitNs) { *abort_p = 1; atomicExch(a.status, SAEM_ERR_TIMEOUT); return -3; }
+            }
+        }
+    };
 
     if (warp == 0) {
         // =============================== producer ===============================
@@ -236,17 +249,11 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         int upcoming = PHASE == 0 || !seam ? (int)blockIdx.x : claim(0);
         for (int n = 0; ok; ++n) {
             const int item = __shfl_sync(0xffffffffu, upcoming, 0);
-            if (item >= total_items) {
-                if (PHASE == 1) {               // tell the MMA warp through the next stage's barrier
-                    ok = mbar_wait(smem_u32(&bar_empty[stage]), phase ^ 1u, abort_p, a.status);
-                    if (ok && lane == 0) {
-                        claimed[n & 15] = -1;
-                        mbar_arrive(smem_u32(&bar_full[stage]));
-                    }
-                }
-                break;
+            if (PHASE == 1 && seam && lane == 0) {
+                claimed[(n + 1) & 15] = -2;          // (its previous user is fifteen items back: nobody reads it any more)
+                claimed[n & 15] = item < total_items ? item : -1;
             }
-            if (PHASE == 1 && lane == 0) claimed[n & 15] = item;
+            if (item >= total_items) break;
             pf_decode(plan, item, cursor, WB, last_cols, it);
             const uint8_t* slot = a.slot_region + (size_t)plan.slot[it.a] * a.slot_bytes;
             // gate/up: chunk (f-block, kc) is 32 KB (gate tile, up tile); down: tiles (2 wb, kc), (2 wb + 1, kc)
@@ -315,21 +322,18 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         PfItem it;
         for (int n = 0; ok; ++n) {
             int item = blockIdx.x + n * G;
-            if (PHASE == 0 && item >= total_items) break;
+            const bool dealt = PHASE == 0 || !seam;      // round-robin: the item is known before its first stage arrives
+            if (dealt) {
+                if (item >= total_items) break;
+                pf_decode(plan, item, cursor, WB, last_cols, it);
+            }
+            if (!dealt) {
+                item = claimed_item(n);
+                if (item < 0) { ok = item == -1; break; }
+                pf_decode(plan, item, cursor, WB, last_cols, it);
+            }
             ok = mbar_wait(smem_u32(&bar_full[stage]), phase, abort_p, a.status);     // the item's first stage
             if (!ok) break;
-            if (PHASE == 1) {                    // which item it is was written before the stage was requested
-                item = claimed[n & 15];
-                if (item < 0) {
-                    // No more items: pass it on to the epilogue warps through the barrier of the accumulator that the next
-                    // tile would have used -- once they have taken that accumulator's previous tile (a barrier must not
-                    // complete two phases before its waiters have seen the first), and behind the MMAs still in flight.
-                    ok = mbar_wait(smem_u32(&bar_acc_empty[acc]), acc_phase[acc] ^ 1u, abort_p, a.status);
-                    if (ok && lane == 0) tc_commit(smem_u32(&bar_acc_full[acc]));
-                    break;
-                }
-            }
-            pf_decode(plan, item, cursor, WB, last_cols, it);
             const int acc0 = acc, acc1 = acc ^ 1;             // accumulators of the item's first / second tile
             const uint32_t idesc = idesc_bf16(it.n_cols);
             for (int kc = 0; ok && kc < KC; ++kc) {
@@ -380,14 +384,18 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
         PfItem it;
         for (int n = 0; ok; ++n) {
             int item = blockIdx.x + n * G;
-            if (PHASE == 0 && item >= total_items) break;
+            const bool dealt = PHASE == 0 || !seam;
+            if (dealt) {
+                if (item >= total_items) break;
+                pf_decode(plan, item, cursor, WB, last_cols, it);
+            }
+            if (!dealt) {
+                item = claimed_item(n);
+                if (item < 0) { ok = item == -1; break; }
+                pf_decode(plan, item, cursor, WB, last_cols, it);
+            }
             ok = mbar_wait(smem_u32(&bar_acc_full[acc]), acc_phase[acc], abort_p, a.status);     // the item's first tile
             if (!ok) break;
-            if (PHASE == 1) {
-                item = claimed[n & 15];
-                if (item < 0) break;
-            }
-            pf_decode(plan, item, cursor, WB, last_cols, it);
             for (int t = 0; ok && t < it.n_mt; ++t) {
                 const int ac = t == 0 ? acc : acc ^ 1;
                 if (t > 0) ok = mbar_wait(smem_u32(&bar_acc_full[ac]), acc_phase[ac], abort_p, a.status);
@@ -488,7 +496,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             }
             if (it.n_mt == 1) acc ^= 1;
             if (PHASE == 0 && seam && ok) {         // this warp's share of the item's h is complete and visible device-wide
-                if (lane == 0) { bulk_wait_all(); fence_proxy_async_all(); }
+                if (lane == 0) bulk_wait_all();          // the tile stores (async proxy) are complete
                 __threadfence();
                 __syncwarp();
                 if (lane == 0) atomicAdd(h_ready + plan.eid[it.a], it.rows_here);
