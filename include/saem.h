@@ -237,7 +237,7 @@ int saem_moe_step_host(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const flo
  * inspection by tests: 0 topk_idx, 1 topk_w, 2 counts, 3 offsets, 4 perm, 5 inv_perm, 6 x_packed,
  * 7 y_packed, 8 shared_y, 9 h (hidden activations), 10 the 656 int32 counters through which the FFN
  * kernels' CTAs meet (arrivals at items whose reduction is split across CTAs; per expert, the hidden
- * activations completed by the gate/up launch and seen by the down launch; the down launch's item
+ * activations completed by the gate/up launch and seen by the down launch, the down launch's item
  * counter): all zero between calls.  NULL for an unknown id.  The one-launch form of
  * the step (see saem_moe_step) does not produce x_packed. */
 void* saem_step_buffer(saem_ctx* ctx, int which);
