@@ -287,7 +287,9 @@ def roofline_of(lb, step_ms, ffn_ms, peaks, which):
                 "frac_of_sustained": achieved / float(peaks.get("bf16_tflops_sustained", 1400.0)),
                 "kernel": "saem_expert_ffn (ffn_prefill_kernel<0/1>: tiled tcgen05 gate/up + down)"}
     else:
-        single = T <= 4 and cfg.top_k <= 8 and lb.layer.shared is None
+        n0 = lb.layer.launches()                 # does saem_moe_step take its one-launch form here?  Count its launches
+        lb.step(0)
+        single = T <= 8 and lb.layer.launches() - n0 <= 2
         ms = step_ms if single else ffn_ms
         nbytes = lb.mean_active_bytes()
         achieved = nbytes / (ms * 1e-3) / 1e9

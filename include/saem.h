@@ -82,7 +82,8 @@ enum { SAEM_FFN_AUTO = 0, SAEM_FFN_SCALAR = 1, SAEM_FFN_TENSOR = 2, SAEM_FFN_TEN
  * rows in the call); SAEM_FFN_TENSOR_PAIRS is SAEM_FFN_TENSOR with the pair form whenever
  * d_model % 256 == 0 (for tests and measurements).  SAEM_FFN_DECODE_FUSED is SAEM_FFN_AUTO, except that
  * saem_moe_step takes its one-launch form (see there) for every batch it supports (up to 8 tokens, top_k
- * up to 8) instead of up to 4 tokens.
+ * up to 8); AUTO takes it up to 4 tokens, and up to 8 on layers whose experts are at most 20 MB
+ * (3 * d_model * d_ff * 2 bytes) and numerous enough (see saem_moe_step).
  * n_shared (0..16, n_experts + n_shared <= SAEM_MAX_EXPERTS): always-on shared experts of the same
  * width d_ff that run INSIDE the layer's grouped launch.  They are experts n_experts ..
  * n_experts + n_shared - 1 of every layer for the cache calls (outside the routed cache-ratio
@@ -215,7 +216,8 @@ int saem_combine(saem_ctx* ctx, const float* y_packed, const int32_t* inv_perm, 
  * holds an always-on shared expert whose width is not a multiple of d_ff (otherwise use
  * config.n_shared and pass NULL).
  * logits[T, E] fp32, x[T, d] bf16, out[T, d] (all dev).
- * Smallest decode batches (ffn_path AUTO: T <= 4, DECODE_FUSED: T <= 8; top_k <= 8; no shared_ctx): the whole step runs as ONE
+ * Smallest decode batches (ffn_path DECODE_FUSED: T <= 8; AUTO: T <= 4, and T <= 8 when an expert is at most 20 MB and
+ * (min(n_experts, T * top_k) + n_shared) * d_model / 32 >= 8 * the device's SM count; top_k <= 8; no shared_ctx): the whole step runs as ONE
  * kernel launch -- gate, repack indices and gate/up projection, a grid-wide barrier, down projection and
  * merge -- launched cooperatively (two launches where the device refuses that).  topk_idx, topk_w, counts,
  * offsets, perm, inv_perm, h and y_packed are still left in the workspace; x_packed is not produced.  A

@@ -461,8 +461,19 @@ int saem_moe_step(saem_ctx* c, saem_ctx* sh, int layer, const float* logits, con
     bool host_mapped = false;
     if (layer >= 0 && layer < g.n_layers)
         for (int e = 0; e < c->n_total; ++e) host_mapped = host_mapped || c->host_of[(size_t)layer * c->n_total + e] != nullptr;
+    // SAEM_FFN_AUTO takes the one-launch form up to 4 tokens, and up to 8 where it was measured ahead of the five
+    // launches: experts of at most 20 MB (a short step, of which the launches' fixed costs are a visible part; the
+    // ERNIE shape's 23.6 MB experts tie, the Mixtral shape's 352 MB lose 5 %) and enough (expert, 32 columns) units in
+    // the down projection for the even unit-major deal (fewer are dealt whole, some CTAs one more than others).
+    bool auto_fused = T <= kDecodeFusedAutoTokens;
+    if (!auto_fused && T <= 8) {
+        const long long expert_bytes = 3ll * g.d_model * g.d_ff * 2;
+        const long long pairs = (long long)T * g.top_k;
+        const long long units = ((pairs < g.n_experts ? pairs : g.n_experts) + g.n_shared) * (g.d_model / 32);
+        auto_fused = expert_bytes <= 20ll * 1024 * 1024 && units >= 8ll * c->n_sm;
+    }
     if (!sh && !host_mapped && decode_fused_supported(T, g.top_k) &&
-        (g.ffn_path == SAEM_FFN_DECODE_FUSED || (g.ffn_path == SAEM_FFN_AUTO && T <= kDecodeFusedAutoTokens))) {
+        (g.ffn_path == SAEM_FFN_DECODE_FUSED || (g.ffn_path == SAEM_FFN_AUTO && auto_fused))) {
         // The smallest decode batches: one launch for the whole step (gate + repack indices + gate/up,
         // grid barrier, down + merge); x_packed is not produced.
         if (layer < 0 || layer >= g.n_layers) return SAEM_ERR_INVALID_ARG;

@@ -54,6 +54,22 @@ def test_single_launch_decode_step_full_shapes(oracle, name, T):
     layer.close()
 
 
+@pytest.mark.parametrize("name,T,one_launch", [("qwen3", 8, True), ("c4", 6, True), ("ernie", 8, False), ("c5", 8, False),
+                                               ("qwen3", 9, False), ("c5", 4, True)])
+def test_default_path_one_launch_range(oracle, name, T, one_launch):
+    """SAEM_FFN_AUTO: saem_moe_step is one launch up to 4 tokens on every layer, and up to 8 tokens on
+    layers of many small experts (at most 20 MB each); five launches otherwise.  Either way the step
+    agrees with the oracle."""
+    import gpu_util as g
+    li = gen.layer_inputs(gen.layer_config(name, tokens=T), n_distinct_experts=4)
+    layer = g.make_layer(li, 0)
+    n0 = layer.launches()
+    g.run_single_call_and_compare(layer, li, oracle)
+    n = layer.launches() - n0
+    assert (n in (1, 2)) if one_launch else n >= 5
+    layer.close()
+
+
 PAIRS = 3       # SAEM_FFN_TENSOR_PAIRS: the CTA-pair form of the tiled kernels wherever the shape allows
 
 
