@@ -49,7 +49,7 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM bytes (read + write) of the two expert-FFN kernels of one step of workload c2 at 16 tokens with all
 # 8 experts active, from an ncu capture (not measured by this run)
-NCU_FFN_TRAFFIC = {("c2", 16): (2831455648, "profiles/ffn_prefill_c2_decode.md (ncu capture, dram__bytes_read.sum + dram__bytes_write.sum)")}
+NCU_FFN_TRAFFIC = {("c2", 16): (2831072592, "profiles/ffn_prefill_c2_decode.md (ncu capture, dram__bytes_read.sum + dram__bytes_write.sum)")}
 STUDY = [("c3", 32, None), ("c3", 2048, None), ("c4", 1, None), ("c4", 8, None), ("c4", 64, None), ("c4", 8, "uniform"),
          ("c4", 64, "uniform"), ("qwen3", 1, None), ("qwen3", 8, None)]
 
