@@ -56,6 +56,8 @@ struct PfPlan {
     int total_items;
     int tpi;                // tokens per item: 128 or 256
     int seam;               // the down launch overlaps the gate/up launch's last round (both launches take the same decision)
+    int half_from;          // down launch: active experts from this one on come as items of ONE 128-column block (see the plan)
+    int t1_last;            // 128-token tiles of the last active expert
     int slot[SAEM_MAX_EXPERTS];
     int eid[SAEM_MAX_EXPERTS];      // expert id of the active expert
     int row0[SAEM_MAX_EXPERTS];
@@ -69,19 +71,27 @@ struct PfItem {
     int n_mt;               // 128-token MMA tiles in this item (1 or 2)
 };
 
-// item -> (active expert, weight block, token tile); weight block slowest, token tile fastest
-__device__ __forceinline__ void pf_decode(const PfPlan& plan, int it, int& cursor, int WB, int last_cols, PfItem& o) {
+// item -> (active expert, weight block, token tile); weight block slowest, token tile fastest.  o.wb: gate/up -> the
+// f-block; down -> the item's first 128-column d-block (an item is two of them, or one: the last odd one, and every item
+// of the experts from plan.half_from on)
+__device__ __forceinline__ void pf_decode(const PfPlan& plan, int it, int& cursor, int WB, int last_cols, bool down, PfItem& o) {
     while (cursor + 1 < plan.n_active && plan.item_base[cursor + 1] <= it) ++cursor;
     o.a = cursor;
     const int local = it - plan.item_base[cursor];
     const int tpi = plan.tpi;
     const int m_blocks = (plan.rows[cursor] + tpi - 1) / tpi;
-    o.wb = local / m_blocks;
-    o.mb = local - o.wb * m_blocks;
+    const int blk = local / m_blocks;
+    o.mb = local - blk * m_blocks;
     o.row_start = plan.row0[cursor] + o.mb * tpi;
     const int left = plan.rows[cursor] - o.mb * tpi;
     o.rows_here = left < tpi ? left : tpi;
-    o.n_cols = (o.wb == WB - 1) ? last_cols : 256;
+    if (down && cursor >= plan.half_from) {
+        o.wb = blk;
+        o.n_cols = 128;
+    } else {
+        o.wb = down ? 2 * blk : blk;
+        o.n_cols = (blk == WB - 1) ? last_cols : 256;
+    }
     o.n_mt = o.rows_here > 128 ? 2 : 1;
 }
 
@@ -177,6 +187,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             plan.row0[n] = r0;
             plan.rows[n] = rows;
             plan.item_base[n] = pair ? (base_t2 + t2_inc - t2) * WB : (base_t1 + t1_inc - t1) * WB;
+            if (n == tot_act - 1) plan.t1_last = t1;
         }
         if (tid == 0) {
             plan.item_base[tot_act] = (pair ? tot_t2 : tot_t1) * WB;
@@ -199,6 +210,27 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             const int rest_gu = (int)(((long long)(pair_gu ? tot_t2 : tot_t1) * wb_gu) % G);
             const bool long_segments = 2 * tot_t1 >= 3 * tot_act;
             plan.seam = (long long)tot_t1 * wb_down > (long long)G && (long_segments || (rest_gu != 0 && 2 * rest_gu <= G)) ? 1 : 0;
+            plan.half_from = 1 << 30;
+        }
+        __syncthreads();
+        // A single round of down items after a gate/up launch with a small last round (the Mixtral shape at 16 tokens:
+        // 896 gate/up items are six rounds and 8 items; 128 down items of 7 MB): the overlap pays after all if the LAST
+        // expert's down items -- the only ones that have to wait for the gate/up tail -- are cut in two (one 128-column
+        // block each): they then take half as long as the other experts' items, which start 25-35 us earlier, and are
+        // no longer what the launch ends with.  Only while everything still fits one round.
+        if (tid == 0 && !plan.seam && plan.n_active >= 2) {
+            const int G = (int)gridDim.x;
+            const int wb_gu = a.f / kTileRows, wb_down = (a.d / kTileRows + 1) / 2, db = a.d / kTileRows;
+            const int rest_gu = (int)(((long long)tot_t1 * wb_gu) % G);
+            const int items = tot_t1 * wb_down + plan.t1_last * (db - wb_down);
+            if (tot_t1 == plan.n_active && rest_gu != 0 && 2 * rest_gu <= G && items <= G) {      // (one tile per expert: no two-tile items)
+                plan.seam = 1;
+                if (PHASE == 1) {
+                    plan.half_from = plan.n_active - 1;
+                    plan.total_items = items;
+                    plan.item_base[plan.n_active] = items;
+                }
+            }
         }
         __syncthreads();
     }
@@ -254,11 +286,11 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                 claimed[n & 15] = item < total_items ? item : -1;
             }
             if (item >= total_items) break;
-            pf_decode(plan, item, cursor, WB, last_cols, it);
+            pf_decode(plan, item, cursor, WB, last_cols, PHASE == 1, it);
             const uint8_t* slot = a.slot_region + (size_t)plan.slot[it.a] * a.slot_bytes;
             // gate/up: chunk (f-block, kc) is 32 KB (gate tile, up tile); down: tiles (2 wb, kc), (2 wb + 1, kc)
             const uint8_t* w0 = PHASE == 0 ? slot + (size_t)it.wb * KC * kPfStageW
-                                           : slot + (size_t)2 * a.d * a.f * 2 + (size_t)(2 * it.wb) * KC * kTileBytes;
+                                           : slot + (size_t)2 * a.d * a.f * 2 + (size_t)it.wb * KC * kTileBytes;
             const uint8_t* w1 = PHASE == 0 ? w0 + kTileBytes : w0 + (size_t)KC * kTileBytes;
             const size_t w_step = PHASE == 0 ? kPfStageW : kTileBytes;
             const int n_boxes = (it.rows_here + 31) / 32;
@@ -325,12 +357,12 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             const bool dealt = PHASE == 0 || !seam;      // round-robin: the item is known before its first stage arrives
             if (dealt) {
                 if (item >= total_items) break;
-                pf_decode(plan, item, cursor, WB, last_cols, it);
+                pf_decode(plan, item, cursor, WB, last_cols, PHASE == 1, it);
             }
             if (!dealt) {
                 item = claimed_item(n);
                 if (item < 0) { ok = item == -1; break; }
-                pf_decode(plan, item, cursor, WB, last_cols, it);
+                pf_decode(plan, item, cursor, WB, last_cols, PHASE == 1, it);
             }
             ok = mbar_wait(smem_u32(&bar_full[stage]), phase, abort_p, a.status);     // the item's first stage
             if (!ok) break;
@@ -387,12 +419,12 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             const bool dealt = PHASE == 0 || !seam;
             if (dealt) {
                 if (item >= total_items) break;
-                pf_decode(plan, item, cursor, WB, last_cols, it);
+                pf_decode(plan, item, cursor, WB, last_cols, PHASE == 1, it);
             }
             if (!dealt) {
                 item = claimed_item(n);
                 if (item < 0) { ok = item == -1; break; }
-                pf_decode(plan, item, cursor, WB, last_cols, it);
+                pf_decode(plan, item, cursor, WB, last_cols, PHASE == 1, it);
             }
             ok = mbar_wait(smem_u32(&bar_acc_full[acc]), acc_phase[acc], abort_p, a.status);     // the item's first tile
             if (!ok) break;
@@ -467,7 +499,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                         }
                     }
                 } else {
-                    float* dst = a.y_packed + row * a.d + (size_t)it.wb * 256 + half * c_half;
+                    float* dst = a.y_packed + row * a.d + (size_t)it.wb * 128 + half * c_half;
 #pragma unroll
                     for (int bx = 0; bx < 8; ++bx) {          // boxes of 16 y columns
                         if (bx * 16 < c_half) {
@@ -481,7 +513,7 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
                                 fence_proxy_async_smem();
                                 __syncwarp();
                                 if (lane == 0) {
-                                    tma_store_2d(&out_map, it.wb * 256 + half * c_half + 16 * bx, box_row, store_buf);
+                                    tma_store_2d(&out_map, it.wb * 128 + half * c_half + 16 * bx, box_row, store_buf);
                                     bulk_commit();
                                 }
                             } else if (valid) {
