@@ -57,7 +57,6 @@ struct PfPlan {
     int tpi;                // tokens per item: 128 or 256
     int seam;               // the down launch overlaps the gate/up launch's last round (both launches take the same decision)
     int half_from;          // down launch: active experts from this one on come as items of ONE 128-column block (see the plan)
-    int t1_last;            // 128-token tiles of the last active expert
     int slot[SAEM_MAX_EXPERTS];
     int eid[SAEM_MAX_EXPERTS];      // expert id of the active expert
     int row0[SAEM_MAX_EXPERTS];
@@ -187,7 +186,6 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             plan.row0[n] = r0;
             plan.rows[n] = rows;
             plan.item_base[n] = pair ? (base_t2 + t2_inc - t2) * WB : (base_t1 + t1_inc - t1) * WB;
-            if (n == tot_act - 1) plan.t1_last = t1;
         }
         if (tid == 0) {
             plan.item_base[tot_act] = (pair ? tot_t2 : tot_t1) * WB;
@@ -195,41 +193,38 @@ ffn_prefill_kernel(FfnArgs a, const __grid_constant__ SlotTable tab, const __gri
             plan.total_items = (pair ? tot_t2 : tot_t1) * WB;
             plan.tpi = pair ? 256 : 128;
             // Do the two launches overlap at their seam?  (Both launches take this decision, from the same numbers.)
-            //  * Not when the down projection is a single round of items (the Mixtral shape at 16 tokens: 128 items of
-            //    7 MB): the items that wait for the last expert's h are as long as the whole launch, nothing is gained
-            //    and the shared bandwidth stretches the gate/up tail (measured 1 % slower).
             //  * When the segments are long (prefill: the SMs that the gate/up launch's last round leaves idle are idle
-            //    tensor pipes), always.
+            //    tensor pipes), always -- given more than one round of down items.
             //  * When they are short (decode: weight streaming) only if that last round occupies at most half of the SMs:
             //    a fuller round keeps HBM busy by itself, and the overlap's bookkeeping then costs more than the idle SMs
-            //    could have fetched (c3 at 32 tokens, 106 of 148 SMs in the last round: 1 % slower with the overlap; the
-            //    Qwen3 shape at 16 tokens, 64 of 148: 5 % faster).
-            const int G = (int)gridDim.x;
-            const int wb_gu = a.f / kTileRows, wb_down = (a.d / kTileRows + 1) / 2;
-            const bool pair_gu = 2ll * tot_t2 * wb_gu >= (long long)kPfPairHalfRounds * G && 2 * tot_t1 >= 3 * tot_t2;
-            const int rest_gu = (int)(((long long)(pair_gu ? tot_t2 : tot_t1) * wb_gu) % G);
-            const bool long_segments = 2 * tot_t1 >= 3 * tot_act;
-            plan.seam = (long long)tot_t1 * wb_down > (long long)G && (long_segments || (rest_gu != 0 && 2 * rest_gu <= G)) ? 1 : 0;
-            plan.half_from = 1 << 30;
-        }
-        __syncthreads();
-        // A single round of down items after a gate/up launch with a small last round (the Mixtral shape at 16 tokens:
-        // 896 gate/up items are six rounds and 8 items; 128 down items of 7 MB): the overlap pays after all if the LAST
-        // expert's down items -- the only ones that have to wait for the gate/up tail -- are cut in two (one 128-column
-        // block each): they then take half as long as the other experts' items, which start 25-35 us earlier, and are
-        // no longer what the launch ends with.  Only while everything still fits one round.
-        if (tid == 0 && !plan.seam && plan.n_active >= 2) {
+            //    could have fetched (c3 at 32 tokens with 106 of 148 SMs in the last round: 1 % slower with the overlap;
+            //    the Qwen3 shape at 16 tokens, 64 of 148: 7 % faster).  The routing decides this step by step.
+            //  * A single round of down items (the Mixtral shape at 16 tokens: 896 gate/up items are six rounds and 8
+            //    items; 128 down items of 7 MB): the items that wait for the last expert's h are as long as the whole
+            //    launch, and overlapping as such gains nothing (measured 1 % slower).  It pays if the LAST expert's down
+            //    items -- the only ones that have to wait for the gate/up tail -- are cut in two (one 128-column block
+            //    each): they are then no longer what the launch ends with.  Only with one token tile per expert and while
+            //    everything still fits one round.
+            // (32-bit arithmetic: at most 65535 rows and 128 weight blocks.)
             const int G = (int)gridDim.x;
             const int wb_gu = a.f / kTileRows, wb_down = (a.d / kTileRows + 1) / 2, db = a.d / kTileRows;
-            const int rest_gu = (int)(((long long)tot_t1 * wb_gu) % G);
-            const int items = tot_t1 * wb_down + plan.t1_last * (db - wb_down);
-            if (tot_t1 == plan.n_active && rest_gu != 0 && 2 * rest_gu <= G && items <= G) {      // (one tile per expert: no two-tile items)
+            const bool pair_gu = 2 * tot_t2 * wb_gu >= kPfPairHalfRounds * G && 2 * tot_t1 >= 3 * tot_t2;
+            const int rest_gu = ((pair_gu ? tot_t2 : tot_t1) * wb_gu) % G;
+            const bool small_rest = rest_gu != 0 && 2 * rest_gu <= G;
+            const bool long_segments = 2 * tot_t1 >= 3 * tot_act;
+            const int items_split = tot_t1 * wb_down + (db - wb_down);
+            plan.half_from = 1 << 30;
+            if (tot_t1 * wb_down > G) {
+                plan.seam = long_segments || small_rest ? 1 : 0;
+            } else if (tot_act >= 2 && tot_t1 == tot_act && small_rest && items_split <= G) {
                 plan.seam = 1;
                 if (PHASE == 1) {
-                    plan.half_from = plan.n_active - 1;
-                    plan.total_items = items;
-                    plan.item_base[plan.n_active] = items;
+                    plan.half_from = tot_act - 1;
+                    plan.total_items = items_split;
+                    plan.item_base[tot_act] = items_split;
                 }
+            } else {
+                plan.seam = 0;
             }
         }
         __syncthreads();
