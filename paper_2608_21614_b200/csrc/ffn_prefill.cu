@@ -30,8 +30,10 @@
 //     epilogue warps advance item by item.  Experts complete in ascending order, so only the items
 //     of the last expert ever wait.  The counts are put back to zero by their last reader.  (Only
 //     where it pays -- see the plan: more than one round of down items, and long segments or a
-//     gate/up launch whose last round leaves at least half of the SMs idle; otherwise the down
-//     launch waits for the gate/up grid as a whole.)
+//     gate/up launch whose last round leaves at least half of the SMs idle; or a single round of
+//     down items of which the last expert's are cut into single 128-column blocks, so that the
+//     items that wait are not what the launch ends with.  Otherwise the down launch waits for the
+//     gate/up grid as a whole.)
 //   * 128 or 256 tokens per item is decided per launch on the device: a stage is released only
 //     when its MMAs have completed and its refill takes about a microsecond, so with 4 x 48 KB
 //     stages of 128-token items the tensor pipe idles about a third of the time; two token tiles
