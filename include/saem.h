@@ -235,6 +235,16 @@ int saem_moe_step(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const float* l
 int saem_moe_step_host(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const float* logits_host,
                        const void* x_host, int T, void* out_host, void* stream);
 
+/*
+ * saem_moe_step_host without the final synchronisation: the two copies in, the kernels and the copy out
+ * are enqueued on `stream` and the call returns.  out_host is valid, and logits_host / x_host may be
+ * reused, once `stream` has passed that point (an event or a synchronisation of the caller's).  Steps
+ * enqueued one after the other run in order; the host's launch work of one overlaps the device's work on
+ * the one before.  Pinned host memory is required for the copies to be asynchronous.
+ */
+int saem_moe_step_host_async(saem_ctx* ctx, saem_ctx* shared_ctx, int layer, const float* logits_host,
+                       const void* x_host, int T, void* out_host, void* stream);
+
 /* Device pointers of the intermediates of the last saem_moe_step (inside the workspace), for
  * inspection by tests: 0 topk_idx, 1 topk_w, 2 counts, 3 offsets, 4 perm, 5 inv_perm, 6 x_packed,
  * 7 y_packed, 8 shared_y, 9 h (hidden activations), 10 the 656 int32 counters through which the FFN

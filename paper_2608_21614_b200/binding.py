@@ -60,6 +60,7 @@ def _load() -> C.CDLL:
         "saem_combine": (i32, [vp, vp, vp, vp, i32, vp, vp, vp]),
         "saem_moe_step": (i32, [vp, vp, i32, vp, vp, i32, vp, vp]),
         "saem_moe_step_host": (i32, [vp, vp, i32, vp, vp, i32, vp, vp]),
+        "saem_moe_step_host_async": (i32, [vp, vp, i32, vp, vp, i32, vp, vp]),
         "saem_step_buffer": (vp, [vp, i32]),
         "saem_cache_load": (i32, [vp, i32, i32, i32, vp, vp]),
         "saem_cache_evict": (i32, [vp, i32, i32]),
@@ -81,7 +82,7 @@ def _load() -> C.CDLL:
 _lib = _load()
 EXPORTS = ("saem_version saem_status_string saem_slot_bytes saem_slot_region_bytes saem_workspace_bytes "
            "saem_create saem_destroy saem_pack_expert_host saem_route saem_route_fused saem_repack saem_expert_ffn saem_combine "
-           "saem_moe_step saem_moe_step_host saem_step_buffer saem_cache_load saem_cache_evict saem_cache_map_host saem_cache_query "
+           "saem_moe_step saem_moe_step_host saem_moe_step_host_async saem_step_buffer saem_cache_load saem_cache_evict saem_cache_map_host saem_cache_query "
            "saem_cache_wait saem_last_device_status saem_launch_count saem_expert_ffn_static saem_selftest_bounded_wait").split()
 
 
@@ -218,6 +219,14 @@ def saem_moe_step_host(ctx, shared_ctx, layer, logits_host, x_host, T, out_host,
                                    _stream(stream))
     if check:
         _check(code, "saem_moe_step_host")
+    return code
+
+
+def saem_moe_step_host_async(ctx, shared_ctx, layer, logits_host, x_host, T, out_host, stream=None, check=True) -> int:
+    code = _lib.saem_moe_step_host_async(ctx, shared_ctx, layer, _ptr(logits_host), _ptr(x_host), T, _ptr(out_host),
+                                         _stream(stream))
+    if check:
+        _check(code, "saem_moe_step_host_async")
     return code
 
 

@@ -506,8 +506,8 @@ int saem_moe_step(saem_ctx* c, saem_ctx* sh, int layer, const float* logits, con
     return saem_combine(c, y, inv, tw, T, sh ? shy : nullptr, out, stream);
 }
 
-int saem_moe_step_host(saem_ctx* c, saem_ctx* sh, int layer, const float* logits_h, const void* x_h, int T,
-                       void* out_h, void* stream) {
+static int step_from_host(saem_ctx* c, saem_ctx* sh, int layer, const float* logits_h, const void* x_h, int T, void* out_h,
+                          void* stream, bool synchronise) {
     int s = check_T(c, T);
     if (s != SAEM_OK) return s;
     if (T == 0) return SAEM_OK;
@@ -522,8 +522,18 @@ int saem_moe_step_host(saem_ctx* c, saem_ctx* sh, int layer, const float* logits
     s = saem_moe_step(c, sh, layer, (const float*)(w + L.logits), w + L.x, T, w + L.out, stream);
     if (s != SAEM_OK) return s;
     CUDA_TRY(cudaMemcpyAsync(out_h, w + L.out, out_bytes, cudaMemcpyDeviceToHost, st));
-    CUDA_TRY(cudaStreamSynchronize(st));
+    if (synchronise) CUDA_TRY(cudaStreamSynchronize(st));
     return SAEM_OK;
+}
+
+int saem_moe_step_host(saem_ctx* c, saem_ctx* sh, int layer, const float* logits_h, const void* x_h, int T, void* out_h,
+                       void* stream) {
+    return step_from_host(c, sh, layer, logits_h, x_h, T, out_h, stream, true);
+}
+
+int saem_moe_step_host_async(saem_ctx* c, saem_ctx* sh, int layer, const float* logits_h, const void* x_h, int T,
+                             void* out_h, void* stream) {
+    return step_from_host(c, sh, layer, logits_h, x_h, T, out_h, stream, false);
 }
 
 // ------------------------------------------------------------------------------------------- cache

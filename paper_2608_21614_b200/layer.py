@@ -140,6 +140,12 @@ class MoELayer:
         B.saem_moe_step_host(self.ctx.handle, self.shared.handle if self.shared else None, layer, logits_host, x_host,
                              T, out_host, stream)
 
+    def step_host_async(self, logits_host: torch.Tensor, x_host: torch.Tensor, T: int, out_host: torch.Tensor,
+                        layer: int = 0, stream=None):
+        """step_host without the final synchronisation: out_host is valid once the stream has passed the call."""
+        B.saem_moe_step_host_async(self.ctx.handle, self.shared.handle if self.shared else None, layer, logits_host,
+                                   x_host, T, out_host, stream)
+
     def device_status(self) -> int:
         s = B.saem_last_device_status(self.ctx.handle)
         if self.shared is not None:

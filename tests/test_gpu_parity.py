@@ -376,6 +376,11 @@ def test_step_calls_agree_bit_for_bit(oracle, fs, merge):
     oh = torch.empty((cfg.tokens, cfg.d_model), dtype=torch.float32).pin_memory()
     layer.step_host(lh, xh, cfg.tokens, oh)
     assert torch.equal(ref_out.cpu(), oh)
+    outs = [torch.zeros_like(oh).pin_memory() for _ in range(3)]      # three steps enqueued without waiting in between
+    for o in outs:
+        layer.step_host_async(lh, xh, cfg.tokens, o)
+    torch.cuda.synchronize()
+    assert all(torch.equal(ref_out.cpu(), o) for o in outs)
     ref = oracle.moe_step(li.logits, li.x, cfg.top_k, li.gate, li.up, li.down, shared=li.shared)
     g.assert_close(oh.numpy(), ref["out"], "out via host call")
     layer.close()
